@@ -1,0 +1,126 @@
+"""Invariants the method fixes, checked on the oracle's whole step (tiny workload)."""
+import copy
+import os
+
+import numpy as np
+
+from paper_1805_10387_b200 import synth
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _build(orc, cfg, init_scale=None, interval=None):
+    layers = [orc.make_layer(synth.weights(cfg, l), cfg.optimizer, cfg.chained(l))
+              for l in range(len(cfg.shapes))]
+    sc = orc.Scaler(init_scale or cfg.init_scale, interval or cfg.growth_interval)
+    opt = orc.Optim(kind=cfg.optimizer, lr=cfg.lr, beta1=cfg.beta1, beta2=cfg.beta2, eps=cfg.eps,
+                    momentum=cfg.momentum)
+    return layers, sc, opt
+
+
+def _inputs(cfg, step):
+    L = len(cfg.shapes)
+    xs = [None if cfg.chained(l) else synth.activations(cfg, l, step) for l in range(L)]
+    gs = [None if cfg.feeds_next(l) else synth.upstream(cfg, l, step) for l in range(L)]
+    return xs, gs
+
+
+def _snapshot(layers):
+    return [(ly.w32.copy(), ly.m.copy(), None if ly.v is None else ly.v.copy(), ly.w16.copy())
+            for ly in layers]
+
+
+def _same(a, b):
+    return all((x is None and y is None) or (x.view(np.uint8) == y.view(np.uint8)).all()
+               for la, lb in zip(a, b) for x, y in zip(la, lb))
+
+
+def test_c1_flags_skip_and_scale_trajectory(orc):
+    cfg = synth.config("c1")
+    layers, sc, opt = _build(orc, cfg)
+    gold = [tuple(int(v) for v in l.split()) for l in open(os.path.join(GOLD, "scaler_c1_trajectory.txt"))
+            if l.strip() and not l.startswith("#")]
+    for step, flag, log2s in gold:
+        before = _snapshot(layers)
+        t_before = sc.t
+        rec = orc.train_step(layers, *_inputs(cfg, step), sc, opt)
+        assert rec.found_inf == flag, step
+        assert rec.S_after == 2.0 ** log2s, step
+        if flag:                                  # overflow step: state bitwise unchanged
+            assert _same(before, _snapshot(layers)) and sc.t == t_before
+        else:
+            assert not _same(before, _snapshot(layers)) and sc.t == t_before + 1
+        for ly in layers:                         # working copy is the rounded master
+            assert (ly.w16 == orc.f2h(ly.w32)).all()
+    assert sc.skipped == 1 and sc.t == 9
+
+
+def _dyadic_inputs(cfg, step):
+    """Inputs on a dyadic grid: X integers in -2..2, upstream gradients multiples of 2^-5 in
+    [-1/4, 1/4].  With weights on a 2^-4 grid every product sum is a multiple of 2^-9, so no
+    nonzero value of the S = 1 run is subnormal in FP16."""
+    rng = np.random.default_rng(100 + step)
+    L = len(cfg.shapes)
+    xs = [None if cfg.chained(l) else
+          synth.fp16_bits(rng.integers(-2, 3, cfg.shapes[l][:2]).astype(np.float32)) for l in range(L)]
+    gs = [None if cfg.feeds_next(l) else
+          (rng.integers(-8, 9, (cfg.shapes[l][0], cfg.shapes[l][2])) / 32.0).astype(np.float32)
+          for l in range(L)]
+    return xs, gs
+
+
+def test_power_of_two_scale_invariance(orc):
+    """With S a power of two and no overflow or underflow, the gradients after unscaling, and
+    so the whole updated state, are bitwise those of the unscaled loss (S = 1)."""
+    cfg = synth.config("c1")
+    rng = np.random.default_rng(1)
+    w_init = [(rng.integers(-4, 5, (k, n)) / 16.0).astype(np.float32) for _, k, n in cfg.shapes]
+    ref = None
+    for k in (0, 1, 5, 8):
+        layers = [orc.make_layer(w_init[l], "adam", cfg.chained(l)) for l in range(2)]
+        sc = orc.Scaler(2.0 ** k, 10 ** 6)
+        rec = orc.train_step(layers, *_dyadic_inputs(cfg, 0), sc, orc.Optim(lr=2.0 ** -10))
+        assert rec.found_inf == 0
+        grads = []
+        for ly in layers:
+            for arr in (ly.dY, ly.dX, ly.dW):             # the premise, checked
+                e = (arr >> 10) & 0x1F
+                assert (e[(arr & 0x7FFF) != 0] > 0).all() and (e < 0x1F).all()
+            grads.append(orc.h2f(ly.dW) * np.float32(2.0 ** -k))
+        snap = _snapshot(layers)
+        if ref is None:
+            ref = (grads, snap)
+        else:
+            assert all((a == b).all() for a, b in zip(ref[0], grads)), k
+            assert _same(ref[1], snap), k
+
+
+def test_static_scale_still_skips_overflow(orc):
+    cfg = synth.config("c1")
+    layers = [orc.make_layer(synth.weights(cfg, l), "adam", cfg.chained(l)) for l in range(2)]
+    sc = orc.Scaler(init_scale=10.0, interval=4, dynamic=False)
+    opt = orc.Optim()
+    for step in range(6):
+        before = _snapshot(layers)
+        rec = orc.train_step(layers, *_inputs(cfg, step), sc, opt)
+        assert rec.S_after == 10.0
+        assert _same(before, _snapshot(layers)) == (step == cfg.inject_inf_step)
+
+
+def test_natural_overflow_halves_until_it_fits(orc):
+    """No injected value: a scale far too large overflows the FP16 gradients by itself, each
+    such step is skipped and halves S, and the first clean step applies."""
+    cfg = synth.config("c1")
+    cfg.inject_inf_step = -1
+    cfg.grad_std = 1.0
+    layers, sc, opt = _build(orc, cfg, init_scale=2.0 ** 16, interval=1000)
+    seen_clean = False
+    for step in range(12):
+        before = _snapshot(layers)
+        rec = orc.train_step(layers, *_inputs(cfg, step), sc, opt)
+        if rec.found_inf:
+            assert not seen_clean and rec.S_after == rec.S_before / 2
+            assert _same(before, _snapshot(layers))
+        else:
+            seen_clean = True
+    assert seen_clean and sc.skipped >= 2
