@@ -1,0 +1,184 @@
+/* mp.h -- C ABI of the mixed-precision training step of a stack of linear layers,
+ * for NVIDIA B200 (sm_100a) only.
+ *
+ * The operations are those of the paper "Mixed-Precision Training for NLP and Speech
+ * Recognition with OpenSeq2Seq" (arXiv 1805.10387), Section 3:
+ *   Section 3.1  matrix products with FP16 operands and FP32 accumulation; a loss scale S
+ *                chosen from an inspection of the gradients and applied to the next step;
+ *                an FP32 master copy of the weights;
+ *   Section 3.2  FP16 gradients converted to FP32, optimizer run on the FP32 master,
+ *                master converted back to the FP16 working copy;
+ *   Section 3.3  weight decay formed from the FP32 master, not from the FP16 copy.
+ *
+ * Conventions
+ *   - Every matrix is row-major.  FP16 means IEEE binary16 stored as 16-bit words.
+ *   - Every tensor pointer is a DEVICE pointer owned by the caller and must be 16-byte
+ *     aligned; leading dimensions (ld*) are in elements and multiples of 8.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  All work is
+ *     asynchronous on that stream; only mp_state_read* synchronise.
+ *   - Every function returns an mp_status.  Nothing throws or aborts.  Argument errors are
+ *     found on the host before anything is launched.  Numeric overflow is NOT an error: it
+ *     is state (found_inf, skipped) held on the device.
+ *   - FP32 -> FP16 conversions round to nearest even, overflow to +-inf (never saturate)
+ *     and keep subnormals.
+ *   - The library owns only mp_state and mp_update_plan objects.  It runs on the device
+ *     that is current when a function is called; objects belong to the device they were
+ *     created on.
+ */
+#ifndef MP_H_
+#define MP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  MP_OK = 0,
+  MP_ERR_INVALID_ARG = -1,      /* null pointer, non-positive size, ld < extent, bad enum  */
+  MP_ERR_ALIGNMENT = -2,        /* pointer not 16-byte aligned or ld not a multiple of 8   */
+  MP_ERR_UNSUPPORTED_ARCH = -3, /* current device is not compute capability 10.x           */
+  MP_ERR_CUDA = -4,             /* a CUDA runtime/driver call failed; see mp_last_error    */
+  MP_ERR_TIMEOUT = -5,          /* a bounded device-side wait expired (reported in status) */
+  MP_ERR_NOMEM = -6,            /* allocation failed or workspace too small                */
+  MP_ERR_TOO_LARGE = -7         /* size beyond a stated maximum                            */
+} mp_status;
+
+typedef struct mp_state mp_state;             /* device-resident scaler + flag + log        */
+typedef struct mp_update_plan mp_update_plan; /* device table over the tensors of an update */
+
+/* Loss-scale policy (Section 3.1, item 1).  dynamic != 0: halve S (not below min_scale) after
+ * a step whose gradients held an inf/NaN, double it (not above max_scale) after
+ * growth_interval clean steps in a row.  dynamic == 0: S stays init_scale (static loss
+ * scaling); an overflow step is still skipped. */
+typedef struct {
+  float init_scale;        /* > 0 */
+  float min_scale;         /* > 0 */
+  float max_scale;         /* >= min_scale */
+  int32_t growth_interval; /* >= 1 */
+  int32_t dynamic;
+} mp_scaler_config;
+
+typedef enum { MP_OPT_ADAM = 0, MP_OPT_MOMENTUM = 1 } mp_opt_kind;
+
+/* Optimizer run on the FP32 master (Section 3.2).  Adam: m = b1 m + (1-b1) g,
+ * v = b2 v + (1-b2) g^2, w -= lr (m/(1-b1^t)) / (sqrt(v/(1-b2^t)) + eps), t = number of
+ * applied steps including this one.  Momentum: u = mu u + g, w -= lr u.
+ * weight_decay adds weight_decay * w32 to g before the moments (Section 3.3). */
+typedef struct {
+  int32_t kind; /* mp_opt_kind */
+  float lr, beta1, beta2, eps, momentum, weight_decay;
+} mp_optim_config;
+
+/* Host copy of the device state, filled by mp_state_read. */
+typedef struct {
+  float scale;         /* S that the NEXT step will use                                     */
+  float min_scale, max_scale;
+  int32_t growth_interval, dynamic;
+  int32_t good_steps;  /* clean steps since S last changed                                  */
+  int32_t found_inf;   /* flag accumulated by the current step so far                       */
+  int32_t status;      /* MP_OK or the first device-side error (MP_ERR_TIMEOUT)             */
+  int64_t t;           /* applied optimizer steps                                           */
+  int64_t step;        /* all steps                                                         */
+  int64_t skipped;     /* overflow steps                                                    */
+} mp_state_host;
+
+/* One record per mp_loss_scale_update call, kept in a device ring of MP_LOG_CAPACITY. */
+typedef struct {
+  int64_t step;
+  int64_t t;           /* after the step */
+  float scale_before, scale_after;
+  int32_t found_inf, good_steps;
+} mp_log_record;
+#define MP_LOG_CAPACITY 4096
+
+/* ---- the five calls of the step ------------------------------------------------------ */
+
+/* Forward product (Section 3.1): Y[M,N] = rn16( sum_k X[m,k] * W[k,n] ), FP32 accumulation.
+ * X16 [M,K] ldx>=K, W16 [K,N] ldw>=N, Y16 [M,N] ldy>=N, all FP16 device buffers.
+ * workspace: device scratch of at least mp_gemm_workspace_bytes(M,K,N,MP_OP_FWD) bytes
+ * (may be NULL when that is 0).  Errors: INVALID_ARG, ALIGNMENT, NOMEM (workspace too
+ * small), UNSUPPORTED_ARCH, CUDA. */
+int mp_linear_fwd(const void* X16, int64_t ldx, const void* W16, int64_t ldw, void* Y16,
+                  int64_t ldy, int64_t M, int64_t K, int64_t N, void* workspace,
+                  size_t workspace_bytes, void* stream);
+
+/* Data gradient (Section 3.2, "gradients are in FP16"): dX[M,K] = rn16( sum_n dY[m,n] *
+ * W[k,n] ).  W is read in place as stored (no transposed copy). */
+int mp_linear_bwd_dgrad(const void* dY16, int64_t lddy, const void* W16, int64_t ldw,
+                        void* dX16, int64_t lddx, int64_t M, int64_t K, int64_t N,
+                        void* workspace, size_t workspace_bytes, void* stream);
+
+/* Weight gradient: dW[K,N] = rn16( sum_m X[m,k] * dY[m,n] ), still multiplied by S.
+ * If state != NULL, state->found_inf is set when any element written to dW16 is inf or NaN
+ * (the gradient inspection of Section 3.1, item 1, done where the gradient is produced). */
+int mp_linear_bwd_wgrad(const void* X16, int64_t ldx, const void* dY16, int64_t lddy,
+                        void* dW16, int64_t lddw, int64_t M, int64_t K, int64_t N,
+                        mp_state* state, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Fused master update over every tensor of the plan (Section 3.2): if the step's flag is
+ * clear, g = float(g16) * (1/S), optimizer on w32 (and m, v), w16 = rn16(w32); if it is set,
+ * nothing is written.  check_mode 0: trust state->found_inf as set by the wgrad calls;
+ * check_mode 1: first inspect every g16 of the plan (sets state->found_inf), then update.
+ * S, t and the flag are read on the device; nothing returns to the host. */
+int mp_master_update(mp_update_plan* plan, mp_state* state, const mp_optim_config* opt,
+                     int check_mode, void* stream);
+
+/* Loss-scale state machine (Section 3.1, item 1: the scale for the next step is chosen from
+ * this step's inspection).  Flag set: S = max(S/2, min_scale), good = 0, skipped++.
+ * Flag clear: t++, good++, and when good == growth_interval: S = min(2S, max_scale), good = 0.
+ * Then the flag is cleared, step++ and a log record is appended.  One tiny kernel. */
+int mp_loss_scale_update(mp_state* state, void* stream);
+
+/* ---- auxiliaries --------------------------------------------------------------------- */
+
+enum { MP_OP_FWD = 0, MP_OP_DGRAD = 1, MP_OP_WGRAD = 2 };
+
+/* Scratch bytes the GEMM of `op` needs for these sizes (0 when it needs none). */
+size_t mp_gemm_workspace_bytes(int64_t M, int64_t K, int64_t N, int op);
+
+/* dY16[i] = rn16( S * g32[i] ), S read from the device state (Section 3.1, item 1: the loss
+ * is scaled; for a linear stack that is the gradient entering the top layer). */
+int mp_scale_upstream(const float* g32, void* dY16, int64_t n, const mp_state* state,
+                      void* stream);
+
+/* Sets state->found_inf if any of the n FP16 values at g16 is inf or NaN. */
+int mp_check_finite(const void* g16, int64_t n, mp_state* state, void* stream);
+
+int mp_state_create(const mp_scaler_config* cfg, mp_state** out);
+int mp_state_destroy(mp_state* state); /* NULL is accepted */
+/* Synchronises `stream`, then copies the device state to *out. */
+int mp_state_read(mp_state* state, mp_state_host* out, void* stream);
+/* Overwrites the device state (resume from a checkpoint); synchronises `stream`. */
+int mp_state_write(mp_state* state, const mp_state_host* in, void* stream);
+/* Copies up to max_records of the most recent log records, oldest first, to out (host);
+ * *n_out receives the count.  Synchronises `stream`. */
+int mp_state_read_log(mp_state* state, mp_log_record* out, int max_records, int* n_out,
+                      void* stream);
+
+/* Plan over n tensors: g16[i], w16[i] FP16 and w32[i], m[i], v[i] FP32 device buffers of
+ * count[i] elements each (count[i] == 0 is legal and skipped).  v may be NULL for a plan
+ * used only with momentum (m then holds the momentum buffer).  The pointer arrays are host
+ * arrays and are copied; the tensors stay the caller's. */
+int mp_update_plan_create(int n, void* const* g16, void* const* w32, void* const* m,
+                          void* const* v, void* const* w16, const int64_t* count,
+                          mp_update_plan** out);
+int mp_update_plan_destroy(mp_update_plan* plan); /* NULL is accepted */
+
+/* Synchronises the device and reports in *out the first device-side error recorded by a GEMM
+ * kernel since the last call (MP_OK, or MP_ERR_TIMEOUT when a bounded wait on a pipeline
+ * barrier expired; the kernel then skipped its remaining work and returned).  Clears it. */
+int mp_gemm_device_status(int* out);
+
+/* Message of the last error on the calling thread ("" if none). */
+const char* mp_last_error(void);
+
+/* Number of kernels this library has launched in the calling process (for accounting). */
+int64_t mp_kernel_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MP_H_ */

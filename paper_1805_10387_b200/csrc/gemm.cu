@@ -1,0 +1,520 @@
+// FP16-in / FP32-accumulate matrix products of the step (Section 3.1 of the paper) as one
+// persistent, warp-specialised tcgen05 kernel for sm_100a:
+//
+//   warp 0      TMA producer: tensor-map loads into a 4-stage shared-memory ring
+//   warp 1      MMA issuer: tcgen05.mma (128x256x16, FP16 x FP16 -> FP32) into tensor memory;
+//               owns the TMEM allocation (two 256-column accumulators, so the epilogue of one
+//               tile overlaps the main loop of the next)
+//   warps 2-5   epilogue: tcgen05.ld, round to FP16 (nearest even, overflow to inf), store;
+//               for the weight gradient also the inf/NaN inspection of what is stored
+//
+// The three products differ only in which operand dimension is contiguous in memory:
+//   forward   Y  = X  * W      A = X  (reduction contiguous)   B = W  (output dim contiguous)
+//   dgrad     dX = dY * W^T    A = dY (reduction contiguous)   B = W  (reduction contiguous)
+//   wgrad     dW = X^T * dY    A = X  (output dim contiguous)  B = dY (output dim contiguous)
+// and that is expressed by the TMA box shape and the "major" bits of the MMA descriptors:
+// no operand is ever transposed in memory.
+//
+// A long reduction with few output tiles (the weight gradient) can be split across CTAs:
+// each split stores FP32 partial sums to a workspace and a second kernel adds them in a
+// fixed order, rounds to FP16 and inspects.
+
+#include <cuda.h>
+#include <cudaTypedefs.h>
+#include <cuda_fp16.h>
+
+#include "common.h"
+#include "ptx.cuh"
+
+namespace {
+
+constexpr int BM = 128, BN = 256, BK = 64, UMMA_K = 16;
+constexpr int STAGES = 4;
+constexpr int A_BYTES = BM * BK * 2;           // 16 KiB
+constexpr int B_BYTES = BN * BK * 2;           // 32 KiB
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int CHUNK_BYTES = 64 * BK * 2;       // one 64 x 64 box of an MN-major operand
+constexpr int THREADS = 192;
+constexpr int TMEM_COLS = 512;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int kModelSMs = 148;                 // used by the split heuristic only
+
+__device__ int g_gemm_status = 0;              // first device-side error (bounded wait expired)
+
+enum OutMode { OUT_F16 = 0, OUT_F16_FLAG = 1, OUT_PARTIAL = 2 };
+
+struct GemmParams {
+  int Mo, No, R;        // output rows, output columns, reduction length
+  int m_tiles, n_tiles, splits, num_kb;
+  int out_mode;
+  uint16_t* out;        // FP16 output [Mo, No], leading dimension ldo
+  int64_t ldo;
+  float* ws;            // FP32 partials [splits][Mo][ws_ld]
+  int64_t ws_ld;
+  int* flag;            // found_inf word, or null
+};
+
+struct Barriers {
+  uint64_t full[STAGES];
+  uint64_t empty[STAGES];
+  uint64_t tmem_full[2];
+  uint64_t tmem_empty[2];
+  uint32_t tmem_base;
+  volatile uint32_t abort;
+};
+
+__device__ __forceinline__ uint32_t pair_nonfinite(uint32_t w) {
+  return __vcmpeq2(w & 0x7C007C00u, 0x7C007C00u);
+}
+
+__device__ __forceinline__ void report_timeout(Barriers* bars) {
+  bars->abort = 1;
+  atomicCAS(&g_gemm_status, 0, (int)MP_ERR_TIMEOUT);
+}
+
+template <bool A_MN, bool B_MN>
+__global__ void __launch_bounds__(THREADS, 1)
+mp_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+               const GemmParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
+                                             ~static_cast<uintptr_t>(1023));
+  Barriers* bars = reinterpret_cast<Barriers*>(smem + STAGES * STAGE_BYTES);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      ptx::mbar_init(&bars->full[s], 1);
+      ptx::mbar_init(&bars->empty[s], 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      ptx::mbar_init(&bars->tmem_full[a], 1);
+      ptx::mbar_init(&bars->tmem_empty[a], 128);
+    }
+    bars->abort = 0;
+    ptx::fence_mbar_init();
+    ptx::prefetch_tensormap(&map_a);
+    ptx::prefetch_tensormap(&map_b);
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc(&bars->tmem_base, TMEM_COLS);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  ptx::tc_fence_after_sync();
+  const uint32_t tmem_base = bars->tmem_base;
+
+  const int total_work = p.m_tiles * p.n_tiles * p.splits;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    int stage = 0;
+    uint32_t phase = 0;
+    int issued = 0;
+    bool ok = true;
+    for (int w = blockIdx.x; w < total_work && ok; w += gridDim.x) {
+      const int split = w % p.splits, tile = w / p.splits;
+      const int m0 = (tile / p.n_tiles) * BM, n0 = (tile % p.n_tiles) * BN;
+      const int kb0 = (int)((int64_t)split * p.num_kb / p.splits);
+      const int kb1 = (int)((int64_t)(split + 1) * p.num_kb / p.splits);
+      for (int kb = kb0; kb < kb1; ++kb) {
+        if (!ptx::mbar_wait(&bars->empty[stage], phase ^ 1)) { ok = false; break; }
+        if (lane == 0) {
+          uint8_t* sA = smem + stage * STAGE_BYTES;
+          uint8_t* sB = sA + A_BYTES;
+          ptx::mbar_arrive_expect_tx(&bars->full[stage], STAGE_BYTES);
+          const int k = kb * BK;
+          if (A_MN) {
+#pragma unroll
+            for (int c = 0; c < BM / 64; ++c)
+              ptx::tma_load_2d(sA + c * CHUNK_BYTES, &map_a, &bars->full[stage], m0 + 64 * c, k);
+          } else {
+            ptx::tma_load_2d(sA, &map_a, &bars->full[stage], k, m0);
+          }
+          if (B_MN) {
+#pragma unroll
+            for (int c = 0; c < BN / 64; ++c)
+              ptx::tma_load_2d(sB + c * CHUNK_BYTES, &map_b, &bars->full[stage], n0 + 64 * c, k);
+          } else {
+            ptx::tma_load_2d(sB, &map_b, &bars->full[stage], k, n0);
+          }
+        }
+        __syncwarp();
+        ++issued;
+        if (++stage == STAGES) { stage = 0; phase ^= 1; }
+      }
+    }
+    if (!ok) report_timeout(bars);
+    if (!ok || bars->abort) {
+      // Leaving early: wait (bounded) until the loads already issued have landed, so that no
+      // copy is in flight into this CTA's shared memory when it exits.
+      const int pending = issued < STAGES ? issued : STAGES;
+      for (int i = 0; i < pending; ++i) {
+        if (--stage < 0) { stage = STAGES - 1; phase ^= 1; }
+        ptx::mbar_wait(&bars->full[stage], phase);
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
+    constexpr uint32_t idesc = ptx::idesc_f16_f32(BM, BN, A_MN, B_MN);
+    int stage = 0;
+    uint32_t phase = 0;
+    int iter = 0;
+    bool ok = true;
+    for (int w = blockIdx.x; w < total_work && ok; w += gridDim.x, ++iter) {
+      const int split = w % p.splits;
+      const int kb0 = (int)((int64_t)split * p.num_kb / p.splits);
+      const int kb1 = (int)((int64_t)(split + 1) * p.num_kb / p.splits);
+      const int acc = iter & 1;
+      const uint32_t acc_phase = (iter >> 1) & 1;
+      if (!ptx::mbar_wait(&bars->tmem_empty[acc], acc_phase ^ 1)) { ok = false; break; }
+      ptx::tc_fence_after_sync();
+      const uint32_t d_tmem = tmem_base + acc * BN;
+      for (int kb = kb0; kb < kb1; ++kb) {
+        if (!ptx::mbar_wait(&bars->full[stage], phase)) { ok = false; break; }
+        ptx::tc_fence_after_sync();
+        if (lane == 0) {
+          const uint32_t sA = ptx::smem_u32(smem + stage * STAGE_BYTES);
+          const uint32_t sB = sA + A_BYTES;
+#pragma unroll
+          for (int kk = 0; kk < BK / UMMA_K; ++kk) {
+            // K-major operand: rows of 128 B, 8-row groups 1024 B apart, a K step of 16
+            // elements is 32 B inside the swizzled row.  MN-major operand: 64-element column
+            // blocks 8 KiB apart (leading offset), 8 reduction rows per 1024 B (stride
+            // offset), a K step of 16 rows is 2 KiB.
+            const uint64_t da = A_MN ? ptx::smem_desc_sw128(sA + kk * 2048, CHUNK_BYTES, 1024)
+                                     : ptx::smem_desc_sw128(sA + kk * 32, 16, 1024);
+            const uint64_t db = B_MN ? ptx::smem_desc_sw128(sB + kk * 2048, CHUNK_BYTES, 1024)
+                                     : ptx::smem_desc_sw128(sB + kk * 32, 16, 1024);
+            ptx::mma_f16_ss(d_tmem, da, db, idesc, (kb > kb0 || kk > 0) ? 1u : 0u);
+          }
+          ptx::mma_commit(&bars->empty[stage]);   // frees the stage when these MMAs are done
+        }
+        __syncwarp();
+        if (++stage == STAGES) { stage = 0; phase ^= 1; }
+      }
+      if (ok && lane == 0) ptx::mma_commit(&bars->tmem_full[acc]);
+      __syncwarp();
+    }
+    if (!ok) report_timeout(bars);
+  } else {
+    // ------------------------------------------------------------ epilogue (warps 2..5)
+    const int q = warp & 3;                         // TMEM lane quarter this warp may read
+    int iter = 0;
+    bool ok = true;
+    for (int w = blockIdx.x; w < total_work && ok; w += gridDim.x, ++iter) {
+      const int split = w % p.splits, tile = w / p.splits;
+      const int m0 = (tile / p.n_tiles) * BM, n0 = (tile % p.n_tiles) * BN;
+      const int acc = iter & 1;
+      const uint32_t acc_phase = (iter >> 1) & 1;
+      if (!ptx::mbar_wait(&bars->tmem_full[acc], acc_phase)) { ok = false; break; }
+      ptx::tc_fence_after_sync();
+      const int row = m0 + q * 32 + lane;
+      const bool row_ok = row < p.Mo;
+      uint32_t bad = 0;
+#pragma unroll 1
+      for (int c = 0; c < BN / 32; ++c) {
+        const int col0 = n0 + c * 32;
+        if (col0 >= p.No) break;                    // warp-uniform
+        uint32_t r[32];
+        ptx::tmem_ld_32x32(tmem_base + acc * BN + c * 32 + ((uint32_t)(q * 32) << 16), r);
+        ptx::tmem_ld_wait();
+        if (p.out_mode == OUT_PARTIAL) {
+          if (row_ok) {
+            float* dst = p.ws + ((int64_t)split * p.Mo + row) * p.ws_ld + col0;
+            if (col0 + 32 <= p.No) {
+#pragma unroll
+              for (int j = 0; j < 8; ++j)
+                *reinterpret_cast<uint4*>(dst + 4 * j) =
+                    make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (col0 + j < p.No) dst[j] = __uint_as_float(r[j]);
+            }
+          }
+        } else {
+          uint32_t h[16];
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const __half2 v = __floats2half2_rn(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1]));
+            h[j] = *reinterpret_cast<const uint32_t*>(&v);
+          }
+          if (row_ok) {
+            uint16_t* dst = p.out + (int64_t)row * p.ldo + col0;
+            if (col0 + 32 <= p.No) {
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                *reinterpret_cast<uint4*>(dst + 8 * j) =
+                    make_uint4(h[4 * j], h[4 * j + 1], h[4 * j + 2], h[4 * j + 3]);
+                bad |= pair_nonfinite(h[4 * j]) | pair_nonfinite(h[4 * j + 1]) |
+                       pair_nonfinite(h[4 * j + 2]) | pair_nonfinite(h[4 * j + 3]);
+              }
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; ++j) {
+                if (col0 + j < p.No) {
+                  const uint16_t hv = (uint16_t)((j & 1) ? (h[j >> 1] >> 16) : (h[j >> 1] & 0xFFFFu));
+                  dst[j] = hv;
+                  bad |= ((hv & 0x7C00u) == 0x7C00u) ? 1u : 0u;
+                }
+              }
+            }
+          }
+        }
+      }
+      if (p.out_mode == OUT_F16_FLAG && p.flag != nullptr) {
+        if (__any_sync(0xFFFFFFFFu, bad != 0) && lane == 0) atomicOr(p.flag, 1);
+      }
+      ptx::tc_fence_before_sync();
+      ptx::mbar_arrive(&bars->tmem_empty[acc]);
+    }
+    if (!ok) report_timeout(bars);
+  }
+
+  // ---------------------------------------------------------------- teardown
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    ptx::tc_fence_after_sync();
+    ptx::tmem_dealloc(tmem_base, TMEM_COLS);
+  }
+}
+
+// Adds the split partial sums in ascending split order, rounds to FP16, stores, inspects.
+__global__ void __launch_bounds__(256)
+mp_splitk_reduce_kernel(const float* __restrict__ ws, int splits, int Mo, int No, int64_t ws_ld,
+                        uint16_t* __restrict__ out, int64_t ldo, int* flag) {
+  const int vec_per_row = (No + 3) / 4;
+  const int64_t total = (int64_t)Mo * vec_per_row;
+  const int64_t split_stride = (int64_t)Mo * ws_ld;
+  uint32_t bad = 0;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total;
+       i += (int64_t)gridDim.x * blockDim.x) {
+    const int row = (int)(i / vec_per_row);
+    const int col = (int)(i % vec_per_row) * 4;
+    const float* src = ws + (int64_t)row * ws_ld + col;
+    if (col + 4 <= No) {
+      float4 acc = *reinterpret_cast<const float4*>(src);
+      for (int s = 1; s < splits; ++s) {
+        const float4 x = *reinterpret_cast<const float4*>(src + s * split_stride);
+        acc.x = __fadd_rn(acc.x, x.x); acc.y = __fadd_rn(acc.y, x.y);
+        acc.z = __fadd_rn(acc.z, x.z); acc.w = __fadd_rn(acc.w, x.w);
+      }
+      const __half2 lo = __floats2half2_rn(acc.x, acc.y), hi = __floats2half2_rn(acc.z, acc.w);
+      const uint2 pk = make_uint2(*reinterpret_cast<const uint32_t*>(&lo),
+                                  *reinterpret_cast<const uint32_t*>(&hi));
+      *reinterpret_cast<uint2*>(out + (int64_t)row * ldo + col) = pk;
+      bad |= pair_nonfinite(pk.x) | pair_nonfinite(pk.y);
+    } else {
+      for (int j = 0; col + j < No; ++j) {
+        float a = src[j];
+        for (int s = 1; s < splits; ++s) a = __fadd_rn(a, src[j + s * split_stride]);
+        const uint16_t hv = __half_as_ushort(__float2half_rn(a));
+        out[(int64_t)row * ldo + col + j] = hv;
+        bad |= ((hv & 0x7C00u) == 0x7C00u) ? 1u : 0u;
+      }
+    }
+  }
+  if (flag != nullptr && __any_sync(0xFFFFFFFFu, bad != 0) && (threadIdx.x & 31) == 0)
+    atomicOr(flag, 1);
+}
+
+// ------------------------------------------------------------------ host side
+PFN_cuTensorMapEncodeTiled_v12000 g_encode = nullptr;
+
+int load_encoder() {
+  if (g_encode) return MP_OK;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  MP_CUDA_TRY(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
+  if (qres != cudaDriverEntryPointSuccess || !fn)
+    return mp::set_error(MP_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
+  g_encode = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(fn);
+  return MP_OK;
+}
+
+// 2-D FP16 tensor map: `inner` contiguous elements per row, `outer` rows, row pitch ld elements.
+int make_map(CUtensorMap* map, const void* ptr, int64_t inner, int64_t outer, int64_t ld,
+             int box_inner, int box_outer) {
+  const cuuint64_t dims[2] = {(cuuint64_t)inner, (cuuint64_t)outer};
+  const cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+  const cuuint32_t box[2] = {(cuuint32_t)box_inner, (cuuint32_t)box_outer};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(ptr), dims,
+                              strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS)
+    return mp::set_error(MP_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
+  return MP_OK;
+}
+
+// Number of reduction splits: minimise a simple time model (waves of tiles on the SMs plus
+// the workspace round trip).  Depends only on the sizes, so that the workspace query and the
+// launch always agree.
+int choose_splits(int64_t Mo, int64_t No, int64_t R) {
+  const int64_t tiles = ((Mo + BM - 1) / BM) * ((No + BN - 1) / BN);
+  const int64_t num_kb = (R + BK - 1) / BK;
+  const double t_kb = 0.42e-6;                   // one 128x256x64 block at ~1.0e13 flop/s per SM
+  const double bw = 4.0e12;                      // workspace traffic, bytes/s
+  int best = 1;
+  double best_t = 1e30;
+  for (int s = 1; s <= 16 && s * 4 <= num_kb; ++s) {
+    const int64_t work = tiles * s;
+    const int64_t waves = (work + kModelSMs - 1) / kModelSMs;
+    double t = (double)waves * (double)((num_kb + s - 1) / s) * t_kb;
+    if (s > 1) t += (double)Mo * (double)No * (8.0 * s + 2.0) / bw + 3e-6;
+    if (t < best_t * 0.97) { best_t = t; best = s; }
+  }
+  return best;
+}
+
+int64_t ws_ld_for(int64_t No) { return (No + 3) / 4 * 4; }
+
+struct Operand {
+  const void* ptr;
+  int64_t ld;
+  bool mn_major;      // true: the output dimension is the contiguous one
+  int64_t mn, red;    // extents along the output dimension and the reduction
+};
+
+template <bool A_MN, bool B_MN>
+int launch(const CUtensorMap& ma, const CUtensorMap& mb, const GemmParams& p, int grid,
+           cudaStream_t st) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    MP_CUDA_TRY(cudaFuncSetAttribute(mp_gemm_kernel<A_MN, B_MN>,
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
+    attr_set = true;
+  }
+  mp_gemm_kernel<A_MN, B_MN><<<grid, THREADS, SMEM_BYTES, st>>>(ma, mb, p);
+  mp::count_launch();
+  MP_CUDA_TRY(cudaGetLastError());
+  return MP_OK;
+}
+
+int run_gemm(const char* name, const Operand& A, const Operand& B, void* out, int64_t ldo,
+             int* flag, bool want_flag, void* workspace, size_t ws_bytes, cudaStream_t st) {
+  const int64_t Mo = A.mn, No = B.mn, R = A.red;
+  if (!A.ptr || !B.ptr || !out) return mp::set_error(MP_ERR_INVALID_ARG, "%s: null pointer", name);
+  if (Mo <= 0 || No <= 0 || R <= 0)
+    return mp::set_error(MP_ERR_INVALID_ARG, "%s: sizes must be positive", name);
+  if (Mo > INT32_MAX / 2 || No > INT32_MAX / 2 || R > INT32_MAX / 2)
+    return mp::set_error(MP_ERR_TOO_LARGE, "%s: a dimension exceeds 2^30", name);
+  const int64_t a_inner = A.mn_major ? A.mn : A.red, b_inner = B.mn_major ? B.mn : B.red;
+  if (A.ld < a_inner || B.ld < b_inner || ldo < No)
+    return mp::set_error(MP_ERR_INVALID_ARG, "%s: leading dimension smaller than the row length", name);
+  if ((A.ld | B.ld | ldo) & 7)
+    return mp::set_error(MP_ERR_ALIGNMENT, "%s: leading dimensions must be multiples of 8", name);
+  if (!mp::aligned16(A.ptr) || !mp::aligned16(B.ptr) || !mp::aligned16(out) ||
+      (workspace && !mp::aligned16(workspace)))
+    return mp::set_error(MP_ERR_ALIGNMENT, "%s: pointers must be 16-byte aligned", name);
+  if (int rc = mp::check_device()) return rc;
+  if (int rc = load_encoder()) return rc;
+
+  GemmParams p;
+  p.Mo = (int)Mo; p.No = (int)No; p.R = (int)R;
+  p.m_tiles = (int)((Mo + BM - 1) / BM);
+  p.n_tiles = (int)((No + BN - 1) / BN);
+  p.num_kb = (int)((R + BK - 1) / BK);
+  p.splits = choose_splits(Mo, No, R);
+  p.out = (uint16_t*)out; p.ldo = ldo;
+  p.ws = (float*)workspace; p.ws_ld = ws_ld_for(No);
+  p.flag = flag;
+  p.out_mode = p.splits > 1 ? OUT_PARTIAL : (want_flag ? OUT_F16_FLAG : OUT_F16);
+  if (p.splits > 1) {
+    const size_t need = (size_t)p.splits * (size_t)Mo * (size_t)p.ws_ld * sizeof(float);
+    if (!workspace || ws_bytes < need)
+      return mp::set_error(MP_ERR_NOMEM, "%s: workspace of %zu bytes needed, %zu given", name, need,
+                           workspace ? ws_bytes : (size_t)0);
+  }
+
+  CUtensorMap ma, mb;
+  if (int rc = A.mn_major ? make_map(&ma, A.ptr, A.mn, A.red, A.ld, 64, BK)
+                          : make_map(&ma, A.ptr, A.red, A.mn, A.ld, BK, BM)) return rc;
+  if (int rc = B.mn_major ? make_map(&mb, B.ptr, B.mn, B.red, B.ld, 64, BK)
+                          : make_map(&mb, B.ptr, B.red, B.mn, B.ld, BK, BN)) return rc;
+
+  int dev = 0, sms = 0;
+  MP_CUDA_TRY(cudaGetDevice(&dev));
+  MP_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+  const int64_t work = (int64_t)p.m_tiles * p.n_tiles * p.splits;
+  const int grid = (int)(work < sms ? work : sms);
+
+  int rc;
+  if (A.mn_major && B.mn_major) rc = launch<true, true>(ma, mb, p, grid, st);
+  else if (!A.mn_major && B.mn_major) rc = launch<false, true>(ma, mb, p, grid, st);
+  else if (!A.mn_major && !B.mn_major) rc = launch<false, false>(ma, mb, p, grid, st);
+  else rc = launch<true, false>(ma, mb, p, grid, st);
+  if (rc) return rc;
+
+  if (p.splits > 1) {
+    const int64_t vecs = Mo * ((No + 3) / 4);
+    int64_t blocks = (vecs + 255) / 256;
+    if (blocks > (int64_t)sms * 8) blocks = (int64_t)sms * 8;
+    mp_splitk_reduce_kernel<<<(int)blocks, 256, 0, st>>>(p.ws, p.splits, p.Mo, p.No, p.ws_ld, p.out,
+                                                         p.ldo, want_flag ? flag : nullptr);
+    mp::count_launch();
+    MP_CUDA_TRY(cudaGetLastError());
+  }
+  return MP_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t mp_gemm_workspace_bytes(int64_t M, int64_t K, int64_t N, int op) {
+  if (M <= 0 || K <= 0 || N <= 0) return 0;
+  int64_t Mo, No, R;
+  if (op == MP_OP_FWD) { Mo = M; No = N; R = K; }
+  else if (op == MP_OP_DGRAD) { Mo = M; No = K; R = N; }
+  else if (op == MP_OP_WGRAD) { Mo = K; No = N; R = M; }
+  else return 0;
+  const int s = choose_splits(Mo, No, R);
+  return s > 1 ? (size_t)s * (size_t)Mo * (size_t)ws_ld_for(No) * sizeof(float) : 0;
+}
+
+int mp_linear_fwd(const void* X16, int64_t ldx, const void* W16, int64_t ldw, void* Y16,
+                  int64_t ldy, int64_t M, int64_t K, int64_t N, void* workspace,
+                  size_t workspace_bytes, void* stream) {
+  const Operand A{X16, ldx, false, M, K};
+  const Operand B{W16, ldw, true, N, K};
+  return run_gemm("mp_linear_fwd", A, B, Y16, ldy, nullptr, false, workspace, workspace_bytes,
+                  (cudaStream_t)stream);
+}
+
+int mp_linear_bwd_dgrad(const void* dY16, int64_t lddy, const void* W16, int64_t ldw,
+                        void* dX16, int64_t lddx, int64_t M, int64_t K, int64_t N,
+                        void* workspace, size_t workspace_bytes, void* stream) {
+  const Operand A{dY16, lddy, false, M, N};
+  const Operand B{W16, ldw, false, K, N};
+  return run_gemm("mp_linear_bwd_dgrad", A, B, dX16, lddx, nullptr, false, workspace,
+                  workspace_bytes, (cudaStream_t)stream);
+}
+
+int mp_linear_bwd_wgrad(const void* X16, int64_t ldx, const void* dY16, int64_t lddy,
+                        void* dW16, int64_t lddw, int64_t M, int64_t K, int64_t N,
+                        mp_state* state, void* workspace, size_t workspace_bytes, void* stream) {
+  const Operand A{X16, ldx, true, K, M};
+  const Operand B{dY16, lddy, true, N, M};
+  int* flag = state ? &state->dev->h.found_inf : nullptr;
+  return run_gemm("mp_linear_bwd_wgrad", A, B, dW16, lddw, flag, state != nullptr, workspace,
+                  workspace_bytes, (cudaStream_t)stream);
+}
+
+// Synchronises the device and returns the first device-side error recorded by a GEMM kernel
+// (MP_OK if none), clearing it.
+int mp_gemm_device_status(int* out) {
+  if (!out) return mp::set_error(MP_ERR_INVALID_ARG, "mp_gemm_device_status: null argument");
+  MP_CUDA_TRY(cudaDeviceSynchronize());
+  int v = 0, zero = 0;
+  MP_CUDA_TRY(cudaMemcpyFromSymbol(&v, g_gemm_status, sizeof(int)));
+  MP_CUDA_TRY(cudaMemcpyToSymbol(g_gemm_status, &zero, sizeof(int)));
+  *out = v;
+  return MP_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,563 @@
+// HBM-streaming kernels of the step: upstream scaling, gradient inspection, the fused
+// unscale + optimizer + FP16 recast over all tensors of a plan, and the loss-scale state
+// machine.  Host entry points for them and for the state / plan objects.
+//
+// Every FP32 operation of the update is written with a round-to-nearest intrinsic so that
+// the compiler cannot contract a multiply and an add into one fused operation: the update
+// is then the sequence of individually rounded operations that Section 3.2 of the paper
+// implies for an FP32 optimizer.  The kernels are bandwidth bound, so this costs nothing.
+
+#include <cuda_fp16.h>
+#include <math.h>
+#include <stdarg.h>
+#include <string.h>
+
+#include <atomic>
+#include <new>
+#include <vector>
+
+#include "common.h"
+
+// ------------------------------------------------------------------ host helpers
+namespace mp {
+
+static thread_local char g_err[512] = "";
+static std::atomic<int64_t> g_launches{0};
+
+int set_error(int code, const char* fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(g_err, sizeof(g_err), fmt, ap);
+  va_end(ap);
+  return code;
+}
+
+void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+int check_device() {
+  int dev = 0;
+  MP_CUDA_TRY(cudaGetDevice(&dev));
+  static thread_local int cached_dev = -1, cached_major = 0;
+  if (cached_dev != dev) {
+    int major = 0;
+    MP_CUDA_TRY(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
+    cached_dev = dev;
+    cached_major = major;
+  }
+  if (cached_major != 10)
+    return set_error(MP_ERR_UNSUPPORTED_ARCH,
+                     "device %d has compute capability %d.x; this library is built for 10.x only",
+                     dev, cached_major);
+  return MP_OK;
+}
+
+}  // namespace mp
+
+// ------------------------------------------------------------------ plan layout
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kVec = 8;                           // elements per 128-bit FP16 vector
+constexpr int kChunk = kThreads * kVec * 2;       // 4096 elements per chunk
+
+struct TensorRec {
+  const uint16_t* g16;
+  float* w32;
+  float* m;
+  float* v;
+  uint16_t* w16;
+  int64_t count;
+};
+
+struct ChunkRec {
+  int32_t tensor;
+  int32_t chunk;  // element offset = chunk * kChunk
+};
+
+struct OptArgs {
+  float lr, b1, b2, eps, mu, wd;
+};
+
+}  // namespace
+
+struct mp_update_plan {
+  TensorRec* d_tensors;
+  ChunkRec* d_chunks;
+  int64_t n_chunks;
+  int64_t total;
+  int n_tensors;
+  int has_v;
+  int device;
+  int sm_count;
+};
+
+namespace {
+
+// ------------------------------------------------------------------ device helpers
+__device__ __forceinline__ uint4 ld_stream_u4(const void* p) {
+  return __ldcs(reinterpret_cast<const uint4*>(p));
+}
+__device__ __forceinline__ float4 ld_stream_f4(const float* p) {
+  return __ldcs(reinterpret_cast<const float4*>(p));
+}
+__device__ __forceinline__ void st_stream_f4(float* p, float4 x) {
+  __stcs(reinterpret_cast<float4*>(p), x);
+}
+__device__ __forceinline__ void st_stream_u4(void* p, uint4 x) {
+  __stcs(reinterpret_cast<uint4*>(p), x);
+}
+
+__device__ __forceinline__ float half_bits_to_float(uint16_t h) {
+  return __half2float(__ushort_as_half(h));
+}
+__device__ __forceinline__ uint16_t float_to_half_bits(float x) {
+  return __half_as_ushort(__float2half_rn(x));  // RNE, overflow -> inf, subnormals kept
+}
+
+// both halves of a packed pair: exponent field all ones <=> inf or NaN
+__device__ __forceinline__ uint32_t pair_nonfinite(uint32_t w) {
+  return __vcmpeq2(w & 0x7C007C00u, 0x7C007C00u);
+}
+
+struct Coef {
+  float inv_s, c1, c2, omb1, omb2;
+};
+
+template <int KIND>
+__device__ __forceinline__ void update_one(float g16f, float& w, float& m, float& v,
+                                           const Coef& c, const OptArgs& o) {
+  float g = __fmul_rn(g16f, c.inv_s);
+  if (o.wd != 0.0f) g = __fadd_rn(g, __fmul_rn(o.wd, w));
+  if (KIND == MP_OPT_ADAM) {
+    m = __fadd_rn(__fmul_rn(o.b1, m), __fmul_rn(c.omb1, g));
+    v = __fadd_rn(__fmul_rn(o.b2, v), __fmul_rn(c.omb2, __fmul_rn(g, g)));
+    const float mh = __fdiv_rn(m, c.c1);
+    const float vh = __fdiv_rn(v, c.c2);
+    w = __fsub_rn(w, __fmul_rn(o.lr, __fdiv_rn(mh, __fadd_rn(__fsqrt_rn(vh), o.eps))));
+  } else {
+    m = __fadd_rn(__fmul_rn(o.mu, m), g);
+    w = __fsub_rn(w, __fmul_rn(o.lr, m));
+  }
+}
+
+template <int KIND>
+__device__ __forceinline__ void update_vec8(const TensorRec& T, int64_t i, const Coef& c,
+                                            const OptArgs& o) {
+  const uint4 gq = ld_stream_u4(T.g16 + i);
+  float4 w0 = ld_stream_f4(T.w32 + i), w1 = ld_stream_f4(T.w32 + i + 4);
+  float4 m0 = ld_stream_f4(T.m + i), m1 = ld_stream_f4(T.m + i + 4);
+  float4 v0 = make_float4(0, 0, 0, 0), v1 = v0;
+  if (KIND == MP_OPT_ADAM) {
+    v0 = ld_stream_f4(T.v + i);
+    v1 = ld_stream_f4(T.v + i + 4);
+  }
+  const uint32_t gw[4] = {gq.x, gq.y, gq.z, gq.w};
+  float* wp[8] = {&w0.x, &w0.y, &w0.z, &w0.w, &w1.x, &w1.y, &w1.z, &w1.w};
+  float* mp_[8] = {&m0.x, &m0.y, &m0.z, &m0.w, &m1.x, &m1.y, &m1.z, &m1.w};
+  float* vp[8] = {&v0.x, &v0.y, &v0.z, &v0.w, &v1.x, &v1.y, &v1.z, &v1.w};
+  uint32_t out[4];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const float g_lo = half_bits_to_float((uint16_t)(gw[j] & 0xFFFFu));
+    const float g_hi = half_bits_to_float((uint16_t)(gw[j] >> 16));
+    update_one<KIND>(g_lo, *wp[2 * j], *mp_[2 * j], *vp[2 * j], c, o);
+    update_one<KIND>(g_hi, *wp[2 * j + 1], *mp_[2 * j + 1], *vp[2 * j + 1], c, o);
+    out[j] = (uint32_t)float_to_half_bits(*wp[2 * j]) |
+             ((uint32_t)float_to_half_bits(*wp[2 * j + 1]) << 16);
+  }
+  st_stream_f4(T.w32 + i, w0);
+  st_stream_f4(T.w32 + i + 4, w1);
+  st_stream_f4(T.m + i, m0);
+  st_stream_f4(T.m + i + 4, m1);
+  if (KIND == MP_OPT_ADAM) {
+    st_stream_f4(T.v + i, v0);
+    st_stream_f4(T.v + i + 4, v1);
+  }
+  st_stream_u4(T.w16 + i, make_uint4(out[0], out[1], out[2], out[3]));
+}
+
+// ------------------------------------------------------------------ kernels
+
+// Fused master update (Section 3.2).  Persistent grid over the plan's chunks; per element
+// 14 B read + 14 B written for Adam, 10 B + 10 B for momentum.  Returns at once, having
+// written nothing, when the step's flag is set.
+template <int KIND>
+__global__ void __launch_bounds__(kThreads)
+mp_master_update_kernel(const TensorRec* __restrict__ tensors, const ChunkRec* __restrict__ chunks,
+                        int64_t n_chunks, const mp_dev_state* __restrict__ st, OptArgs o) {
+  if (*reinterpret_cast<const volatile int32_t*>(&st->h.found_inf) != 0) return;
+  __shared__ Coef s_coef;
+  if (threadIdx.x == 0) {
+    const double t = (double)(st->h.t + 1);  // applied steps including this one
+    Coef c;
+    c.inv_s = __fdiv_rn(1.0f, st->h.scale);
+    c.c1 = (float)(1.0 - pow((double)o.b1, t));
+    c.c2 = (float)(1.0 - pow((double)o.b2, t));
+    c.omb1 = __fsub_rn(1.0f, o.b1);
+    c.omb2 = __fsub_rn(1.0f, o.b2);
+    s_coef = c;
+  }
+  __syncthreads();
+  const Coef c = s_coef;
+  for (int64_t ch = blockIdx.x; ch < n_chunks; ch += gridDim.x) {
+    const ChunkRec rec = chunks[ch];
+    const TensorRec T = tensors[rec.tensor];
+    const int64_t start = (int64_t)rec.chunk * kChunk;
+    const int64_t rem = T.count - start;
+    const int n = rem < kChunk ? (int)rem : kChunk;
+    if (n == kChunk) {
+      update_vec8<KIND>(T, start + threadIdx.x * kVec, c, o);
+      update_vec8<KIND>(T, start + (kThreads + threadIdx.x) * kVec, c, o);
+    } else {
+      const int nvec = n / kVec;
+      for (int q = threadIdx.x; q < nvec; q += kThreads)
+        update_vec8<KIND>(T, start + (int64_t)q * kVec, c, o);
+      const int tail = n - nvec * kVec;  // < 8 elements, past the last full vector
+      if ((int)threadIdx.x < tail) {
+        const int64_t i = start + nvec * kVec + threadIdx.x;
+        float w = T.w32[i], m = T.m[i], v = (KIND == MP_OPT_ADAM) ? T.v[i] : 0.0f;
+        update_one<KIND>(half_bits_to_float(T.g16[i]), w, m, v, c, o);
+        T.w32[i] = w;
+        T.m[i] = m;
+        if (KIND == MP_OPT_ADAM) T.v[i] = v;
+        T.w16[i] = float_to_half_bits(w);
+      }
+    }
+  }
+}
+
+// Gradient inspection over a plan (Section 3.1, item 1): 2 B read per element, OR-reduced
+// by warp vote, at most one atomic per block and only when something was found.
+__global__ void __launch_bounds__(kThreads)
+mp_check_plan_kernel(const TensorRec* __restrict__ tensors, const ChunkRec* __restrict__ chunks,
+                     int64_t n_chunks, mp_dev_state* __restrict__ st) {
+  uint32_t bad = 0;
+  for (int64_t ch = blockIdx.x; ch < n_chunks; ch += gridDim.x) {
+    const ChunkRec rec = chunks[ch];
+    const uint16_t* g = tensors[rec.tensor].g16;
+    const int64_t start = (int64_t)rec.chunk * kChunk;
+    const int64_t rem = tensors[rec.tensor].count - start;
+    const int n = rem < kChunk ? (int)rem : kChunk;
+    const int nvec = n / kVec;
+    for (int q = threadIdx.x; q < nvec; q += kThreads) {
+      const uint4 x = ld_stream_u4(g + start + (int64_t)q * kVec);
+      bad |= pair_nonfinite(x.x) | pair_nonfinite(x.y) | pair_nonfinite(x.z) | pair_nonfinite(x.w);
+    }
+    const int tail = n - nvec * kVec;
+    if ((int)threadIdx.x < tail) {
+      const uint16_t h = g[start + nvec * kVec + threadIdx.x];
+      bad |= ((h & 0x7C00u) == 0x7C00u) ? 1u : 0u;
+    }
+  }
+  const int warp_bad = __any_sync(0xFFFFFFFFu, bad != 0);
+  __shared__ int s_bad;
+  if (threadIdx.x == 0) s_bad = 0;
+  __syncthreads();
+  if (warp_bad && (threadIdx.x & 31) == 0) s_bad = 1;
+  __syncthreads();
+  if (threadIdx.x == 0 && s_bad) atomicOr(&st->h.found_inf, 1);
+}
+
+// Inspection of one flat FP16 buffer.
+__global__ void __launch_bounds__(kThreads)
+mp_check_flat_kernel(const uint16_t* __restrict__ g, int64_t n, mp_dev_state* __restrict__ st) {
+  uint32_t bad = 0;
+  const int64_t nvec = n / kVec;
+  for (int64_t q = (int64_t)blockIdx.x * kThreads + threadIdx.x; q < nvec;
+       q += (int64_t)gridDim.x * kThreads) {
+    const uint4 x = ld_stream_u4(g + q * kVec);
+    bad |= pair_nonfinite(x.x) | pair_nonfinite(x.y) | pair_nonfinite(x.z) | pair_nonfinite(x.w);
+  }
+  if (blockIdx.x == 0 && (int64_t)threadIdx.x < n - nvec * kVec) {
+    const uint16_t h = g[nvec * kVec + threadIdx.x];
+    bad |= ((h & 0x7C00u) == 0x7C00u) ? 1u : 0u;
+  }
+  const int warp_bad = __any_sync(0xFFFFFFFFu, bad != 0);
+  __shared__ int s_bad;
+  if (threadIdx.x == 0) s_bad = 0;
+  __syncthreads();
+  if (warp_bad && (threadIdx.x & 31) == 0) s_bad = 1;
+  __syncthreads();
+  if (threadIdx.x == 0 && s_bad) atomicOr(&st->h.found_inf, 1);
+}
+
+// dY16 = rn16(S * g32), S read on the device (Section 3.1, item 1).
+__global__ void __launch_bounds__(kThreads)
+mp_scale_upstream_kernel(const float* __restrict__ g32, uint16_t* __restrict__ out, int64_t n,
+                         const mp_dev_state* __restrict__ st) {
+  const float S = st->h.scale;
+  const int64_t nvec = n / kVec;
+  for (int64_t q = (int64_t)blockIdx.x * kThreads + threadIdx.x; q < nvec;
+       q += (int64_t)gridDim.x * kThreads) {
+    const float4 a = ld_stream_f4(g32 + q * kVec), b = ld_stream_f4(g32 + q * kVec + 4);
+    uint4 r;
+    r.x = (uint32_t)float_to_half_bits(__fmul_rn(S, a.x)) | ((uint32_t)float_to_half_bits(__fmul_rn(S, a.y)) << 16);
+    r.y = (uint32_t)float_to_half_bits(__fmul_rn(S, a.z)) | ((uint32_t)float_to_half_bits(__fmul_rn(S, a.w)) << 16);
+    r.z = (uint32_t)float_to_half_bits(__fmul_rn(S, b.x)) | ((uint32_t)float_to_half_bits(__fmul_rn(S, b.y)) << 16);
+    r.w = (uint32_t)float_to_half_bits(__fmul_rn(S, b.z)) | ((uint32_t)float_to_half_bits(__fmul_rn(S, b.w)) << 16);
+    *reinterpret_cast<uint4*>(out + q * kVec) = r;
+  }
+  if (blockIdx.x == 0 && (int64_t)threadIdx.x < n - nvec * kVec) {
+    const int64_t i = nvec * kVec + threadIdx.x;
+    out[i] = float_to_half_bits(__fmul_rn(S, g32[i]));
+  }
+}
+
+// Loss-scale state machine, one thread (Section 3.1, item 1).
+__global__ void mp_loss_scale_update_kernel(mp_dev_state* st) {
+  mp_state_host& h = st->h;
+  mp_log_record rec;
+  rec.step = h.step;
+  rec.scale_before = h.scale;
+  rec.found_inf = h.found_inf != 0;
+  if (h.found_inf != 0) {
+    h.skipped += 1;
+    h.good_steps = 0;
+    if (h.dynamic) h.scale = fmaxf(__fmul_rn(h.scale, 0.5f), h.min_scale);
+  } else {
+    h.t += 1;
+    h.good_steps += 1;
+    if (h.dynamic && h.good_steps >= h.growth_interval) {
+      h.scale = fminf(__fmul_rn(h.scale, 2.0f), h.max_scale);
+      h.good_steps = 0;
+    }
+  }
+  h.found_inf = 0;
+  h.step += 1;
+  rec.t = h.t;
+  rec.scale_after = h.scale;
+  rec.good_steps = h.good_steps;
+  st->log[st->log_count % MP_LOG_CAPACITY] = rec;
+  st->log_count += 1;
+}
+
+int grid_for(int64_t work_blocks, int sm_count, int per_sm) {
+  const int64_t cap = (int64_t)sm_count * per_sm;
+  return (int)(work_blocks < cap ? (work_blocks > 0 ? work_blocks : 1) : cap);
+}
+
+int sm_count_of_current_device(int* out) {
+  int dev = 0;
+  MP_CUDA_TRY(cudaGetDevice(&dev));
+  MP_CUDA_TRY(cudaDeviceGetAttribute(out, cudaDevAttrMultiProcessorCount, dev));
+  return MP_OK;
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------ C ABI
+extern "C" {
+
+const char* mp_last_error(void) { return mp::g_err; }
+int64_t mp_kernel_launch_count(void) { return mp::g_launches.load(); }
+
+int mp_state_create(const mp_scaler_config* cfg, mp_state** out) {
+  if (!cfg || !out) return mp::set_error(MP_ERR_INVALID_ARG, "mp_state_create: null argument");
+  if (!(cfg->init_scale > 0) || !(cfg->min_scale > 0) || !(cfg->max_scale >= cfg->min_scale) ||
+      cfg->growth_interval < 1)
+    return mp::set_error(MP_ERR_INVALID_ARG, "mp_state_create: bad scaler configuration");
+  if (int rc = mp::check_device()) return rc;
+  mp_state* s = new (std::nothrow) mp_state{nullptr, 0};
+  if (!s) return mp::set_error(MP_ERR_NOMEM, "mp_state_create: host allocation failed");
+  cudaGetDevice(&s->device);
+  if (cudaMalloc(&s->dev, sizeof(mp_dev_state)) != cudaSuccess) {
+    delete s;
+    return mp::set_error(MP_ERR_NOMEM, "mp_state_create: device allocation failed");
+  }
+  cudaMemset(s->dev, 0, sizeof(mp_dev_state));
+  mp_state_host h;
+  memset(&h, 0, sizeof(h));
+  h.scale = cfg->init_scale;
+  h.min_scale = cfg->min_scale;
+  h.max_scale = cfg->max_scale;
+  h.growth_interval = cfg->growth_interval;
+  h.dynamic = cfg->dynamic ? 1 : 0;
+  cudaError_t e = cudaMemcpy(s->dev, &h, sizeof(h), cudaMemcpyHostToDevice);
+  if (e != cudaSuccess) {
+    cudaFree(s->dev);
+    delete s;
+    return mp::set_error(MP_ERR_CUDA, "mp_state_create: %s", cudaGetErrorString(e));
+  }
+  *out = s;
+  return MP_OK;
+}
+
+int mp_state_destroy(mp_state* s) {
+  if (!s) return MP_OK;
+  cudaFree(s->dev);
+  delete s;
+  return MP_OK;
+}
+
+int mp_state_read(mp_state* s, mp_state_host* out, void* stream) {
+  if (!s || !out) return mp::set_error(MP_ERR_INVALID_ARG, "mp_state_read: null argument");
+  cudaStream_t st = (cudaStream_t)stream;
+  MP_CUDA_TRY(cudaMemcpyAsync(out, s->dev, sizeof(*out), cudaMemcpyDeviceToHost, st));
+  MP_CUDA_TRY(cudaStreamSynchronize(st));
+  return MP_OK;
+}
+
+int mp_state_write(mp_state* s, const mp_state_host* in, void* stream) {
+  if (!s || !in) return mp::set_error(MP_ERR_INVALID_ARG, "mp_state_write: null argument");
+  cudaStream_t st = (cudaStream_t)stream;
+  MP_CUDA_TRY(cudaMemcpyAsync(s->dev, in, sizeof(*in), cudaMemcpyHostToDevice, st));
+  MP_CUDA_TRY(cudaStreamSynchronize(st));
+  return MP_OK;
+}
+
+int mp_state_read_log(mp_state* s, mp_log_record* out, int max_records, int* n_out, void* stream) {
+  if (!s || !out || !n_out || max_records < 0)
+    return mp::set_error(MP_ERR_INVALID_ARG, "mp_state_read_log: bad argument");
+  cudaStream_t st = (cudaStream_t)stream;
+  int64_t total = 0;
+  MP_CUDA_TRY(cudaMemcpyAsync(&total, &s->dev->log_count, sizeof(total), cudaMemcpyDeviceToHost, st));
+  MP_CUDA_TRY(cudaStreamSynchronize(st));
+  int64_t have = total < MP_LOG_CAPACITY ? total : MP_LOG_CAPACITY;
+  if (have > max_records) have = max_records;
+  for (int64_t i = 0; i < have; ++i) {
+    const int64_t idx = (total - have + i) % MP_LOG_CAPACITY;
+    MP_CUDA_TRY(cudaMemcpyAsync(out + i, &s->dev->log[idx], sizeof(mp_log_record),
+                                cudaMemcpyDeviceToHost, st));
+  }
+  MP_CUDA_TRY(cudaStreamSynchronize(st));
+  *n_out = (int)have;
+  return MP_OK;
+}
+
+int mp_update_plan_create(int n, void* const* g16, void* const* w32, void* const* m,
+                          void* const* v, void* const* w16, const int64_t* count,
+                          mp_update_plan** out) {
+  if (n <= 0 || !g16 || !w32 || !m || !w16 || !count || !out)
+    return mp::set_error(MP_ERR_INVALID_ARG, "mp_update_plan_create: null argument or n <= 0");
+  if (int rc = mp::check_device()) return rc;
+  std::vector<TensorRec> recs(n);
+  std::vector<ChunkRec> chunks;
+  int64_t total = 0;
+  for (int i = 0; i < n; ++i) {
+    if (count[i] < 0)
+      return mp::set_error(MP_ERR_INVALID_ARG, "mp_update_plan_create: count[%d] < 0", i);
+    if (count[i] > 0) {
+      if (!g16[i] || !w32[i] || !m[i] || !w16[i] || (v && !v[i]))
+        return mp::set_error(MP_ERR_INVALID_ARG, "mp_update_plan_create: tensor %d has a null buffer", i);
+      if (!mp::aligned16(g16[i]) || !mp::aligned16(w32[i]) || !mp::aligned16(m[i]) ||
+          !mp::aligned16(w16[i]) || (v && !mp::aligned16(v[i])))
+        return mp::set_error(MP_ERR_ALIGNMENT, "mp_update_plan_create: tensor %d is not 16-byte aligned", i);
+    }
+    recs[i] = TensorRec{(const uint16_t*)g16[i], (float*)w32[i], (float*)m[i],
+                        v ? (float*)v[i] : nullptr, (uint16_t*)w16[i], count[i]};
+    const int64_t nch = (count[i] + kChunk - 1) / kChunk;
+    if (nch > INT32_MAX)
+      return mp::set_error(MP_ERR_TOO_LARGE, "mp_update_plan_create: tensor %d is too large", i);
+    for (int64_t c = 0; c < nch; ++c) chunks.push_back(ChunkRec{i, (int32_t)c});
+    total += count[i];
+  }
+  mp_update_plan* p = new (std::nothrow) mp_update_plan();
+  if (!p) return mp::set_error(MP_ERR_NOMEM, "mp_update_plan_create: host allocation failed");
+  memset(p, 0, sizeof(*p));
+  p->n_tensors = n;
+  p->n_chunks = (int64_t)chunks.size();
+  p->total = total;
+  p->has_v = v != nullptr;
+  cudaGetDevice(&p->device);
+  if (int rc = sm_count_of_current_device(&p->sm_count)) { delete p; return rc; }
+  const size_t chunk_bytes = (chunks.size() ? chunks.size() : 1) * sizeof(ChunkRec);
+  if (cudaMalloc(&p->d_tensors, n * sizeof(TensorRec)) != cudaSuccess ||
+      cudaMalloc(&p->d_chunks, chunk_bytes) != cudaSuccess) {
+    cudaFree(p->d_tensors);
+    delete p;
+    return mp::set_error(MP_ERR_NOMEM, "mp_update_plan_create: device allocation failed");
+  }
+  cudaError_t e = cudaMemcpy(p->d_tensors, recs.data(), n * sizeof(TensorRec), cudaMemcpyHostToDevice);
+  if (e == cudaSuccess && !chunks.empty())
+    e = cudaMemcpy(p->d_chunks, chunks.data(), chunks.size() * sizeof(ChunkRec), cudaMemcpyHostToDevice);
+  if (e != cudaSuccess) {
+    mp_update_plan_destroy(p);
+    return mp::set_error(MP_ERR_CUDA, "mp_update_plan_create: %s", cudaGetErrorString(e));
+  }
+  *out = p;
+  return MP_OK;
+}
+
+int mp_update_plan_destroy(mp_update_plan* p) {
+  if (!p) return MP_OK;
+  cudaFree(p->d_tensors);
+  cudaFree(p->d_chunks);
+  delete p;
+  return MP_OK;
+}
+
+int mp_master_update(mp_update_plan* plan, mp_state* state, const mp_optim_config* opt,
+                     int check_mode, void* stream) {
+  if (!plan || !state || !opt)
+    return mp::set_error(MP_ERR_INVALID_ARG, "mp_master_update: null argument");
+  if (opt->kind != MP_OPT_ADAM && opt->kind != MP_OPT_MOMENTUM)
+    return mp::set_error(MP_ERR_INVALID_ARG, "mp_master_update: unknown optimizer kind %d", opt->kind);
+  if (opt->kind == MP_OPT_ADAM && !plan->has_v)
+    return mp::set_error(MP_ERR_INVALID_ARG, "mp_master_update: Adam needs a plan created with v");
+  if (check_mode != 0 && check_mode != 1)
+    return mp::set_error(MP_ERR_INVALID_ARG, "mp_master_update: check_mode must be 0 or 1");
+  if (int rc = mp::check_device()) return rc;
+  if (plan->n_chunks == 0) return MP_OK;
+  cudaStream_t st = (cudaStream_t)stream;
+  const OptArgs o{opt->lr, opt->beta1, opt->beta2, opt->eps, opt->momentum, opt->weight_decay};
+  if (check_mode == 1) {
+    mp_check_plan_kernel<<<grid_for(plan->n_chunks, plan->sm_count, 16), kThreads, 0, st>>>(
+        plan->d_tensors, plan->d_chunks, plan->n_chunks, state->dev);
+    mp::count_launch();
+  }
+  const int grid = grid_for(plan->n_chunks, plan->sm_count, 8);
+  if (opt->kind == MP_OPT_ADAM)
+    mp_master_update_kernel<MP_OPT_ADAM><<<grid, kThreads, 0, st>>>(
+        plan->d_tensors, plan->d_chunks, plan->n_chunks, state->dev, o);
+  else
+    mp_master_update_kernel<MP_OPT_MOMENTUM><<<grid, kThreads, 0, st>>>(
+        plan->d_tensors, plan->d_chunks, plan->n_chunks, state->dev, o);
+  mp::count_launch();
+  MP_CUDA_TRY(cudaGetLastError());
+  return MP_OK;
+}
+
+int mp_loss_scale_update(mp_state* state, void* stream) {
+  if (!state) return mp::set_error(MP_ERR_INVALID_ARG, "mp_loss_scale_update: null state");
+  if (int rc = mp::check_device()) return rc;
+  mp_loss_scale_update_kernel<<<1, 1, 0, (cudaStream_t)stream>>>(state->dev);
+  mp::count_launch();
+  MP_CUDA_TRY(cudaGetLastError());
+  return MP_OK;
+}
+
+int mp_scale_upstream(const float* g32, void* dY16, int64_t n, const mp_state* state, void* stream) {
+  if (!g32 || !dY16 || !state || n < 0)
+    return mp::set_error(MP_ERR_INVALID_ARG, "mp_scale_upstream: bad argument");
+  if (!mp::aligned16(g32) || !mp::aligned16(dY16))
+    return mp::set_error(MP_ERR_ALIGNMENT, "mp_scale_upstream: buffers must be 16-byte aligned");
+  if (int rc = mp::check_device()) return rc;
+  if (n == 0) return MP_OK;
+  int sms = 0;
+  if (int rc = sm_count_of_current_device(&sms)) return rc;
+  const int64_t blocks = (n / kVec + kThreads - 1) / kThreads;
+  mp_scale_upstream_kernel<<<grid_for(blocks, sms, 16), kThreads, 0, (cudaStream_t)stream>>>(
+      g32, (uint16_t*)dY16, n, state->dev);
+  mp::count_launch();
+  MP_CUDA_TRY(cudaGetLastError());
+  return MP_OK;
+}
+
+int mp_check_finite(const void* g16, int64_t n, mp_state* state, void* stream) {
+  if (!g16 || !state || n < 0)
+    return mp::set_error(MP_ERR_INVALID_ARG, "mp_check_finite: bad argument");
+  if (!mp::aligned16(g16))
+    return mp::set_error(MP_ERR_ALIGNMENT, "mp_check_finite: buffer must be 16-byte aligned");
+  if (int rc = mp::check_device()) return rc;
+  if (n == 0) return MP_OK;
+  int sms = 0;
+  if (int rc = sm_count_of_current_device(&sms)) return rc;
+  const int64_t blocks = (n / kVec + kThreads - 1) / kThreads;
+  mp_check_flat_kernel<<<grid_for(blocks, sms, 16), kThreads, 0, (cudaStream_t)stream>>>(
+      (const uint16_t*)g16, n, state->dev);
+  mp::count_launch();
+  MP_CUDA_TRY(cudaGetLastError());
+  return MP_OK;
+}
+
+}  // extern "C"

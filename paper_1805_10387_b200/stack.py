@@ -1,0 +1,123 @@
+"""One mixed-precision training step of a stack of linear layers, as a sequence of calls
+into the C-ABI library.  This module only owns device buffers and orders the calls; it does
+no arithmetic.
+
+Order of one step (paper Section 3.1-3.2): forward products bottom-up; the FP32 gradient
+entering each top layer is multiplied by the current loss scale S on the device; backward
+products top-down (the weight-gradient kernels inspect what they store and raise the
+device flag); one fused master update over all layers, which writes nothing when the flag
+is set; the loss-scale state machine picks S for the next step.  Nothing returns to the
+host inside a step.
+"""
+from __future__ import annotations
+
+import torch
+
+from . import mp
+
+
+def _align(n: int, a: int = 8) -> int:
+    return (n + a - 1) // a * a
+
+
+class LinearStack:
+    def __init__(self, shapes, chained, optimizer="adam", lr=1e-3, beta1=0.9, beta2=0.999,
+                 eps=1e-8, momentum=0.9, weight_decay=0.0, init_scale=65536.0,
+                 growth_interval=1000, min_scale=1.0, max_scale=2.0 ** 24, dynamic=True,
+                 device="cuda"):
+        self.shapes = [tuple(s) for s in shapes]
+        self.chained = list(chained)
+        self.L = len(shapes)
+        self.device = torch.device(device)
+        self.opt = mp.OptimConfig(mp.MP_OPT_ADAM if optimizer == "adam" else mp.MP_OPT_MOMENTUM,
+                                  lr, beta1, beta2, eps, momentum, weight_decay)
+        self.state = mp.State(init_scale, growth_interval, min_scale, max_scale, dynamic)
+
+        # parameters, moments and weight gradients live in flat buffers; every tensor starts on
+        # a 16-byte boundary and rows are padded to a multiple of 8 elements
+        self.ldw = [_align(n) for _, _, n in self.shapes]
+        sizes = [k * ld for (_, k, _), ld in zip(self.shapes, self.ldw)]
+        offs, total = [], 0
+        for s in sizes:
+            offs.append(total)
+            total += _align(s)
+        self.offsets, self.total = offs, total
+        f16 = dict(dtype=torch.float16, device=self.device)
+        f32 = dict(dtype=torch.float32, device=self.device)
+        self.w16_flat = torch.zeros(total, **f16)
+        self.dw_flat = torch.zeros(total, **f16)
+        self.w32_flat = torch.zeros(total, **f32)
+        self.m_flat = torch.zeros(total, **f32)
+        self.v_flat = torch.zeros(total, **f32) if optimizer == "adam" else None
+        view = lambda flat, l: flat[offs[l]:offs[l] + sizes[l]].view(self.shapes[l][1], self.ldw[l])
+        self.w16 = [view(self.w16_flat, l) for l in range(self.L)]
+        self.dw = [view(self.dw_flat, l) for l in range(self.L)]
+        self.w32 = [view(self.w32_flat, l) for l in range(self.L)]
+        self.m = [view(self.m_flat, l) for l in range(self.L)]
+        self.v = [view(self.v_flat, l) for l in range(self.L)] if self.v_flat is not None else None
+        # one plan over the whole flat range: padding columns hold zeros and stay zero
+        self.plan = mp.UpdatePlan([self.dw_flat], [self.w32_flat], [self.m_flat],
+                                  [self.v_flat] if self.v_flat is not None else None,
+                                  [self.w16_flat])
+
+        # activations and their gradients
+        self.x = [None] * self.L
+        self.y = [torch.empty(m, _align(n), **f16) for m, _, n in self.shapes]
+        self.dy = [None] * self.L
+        self.dx = [torch.empty(m, _align(k), **f16) for m, k, _ in self.shapes]
+        for l in range(self.L):
+            if self.chained[l]:
+                self.x[l] = self.y[l - 1]
+            feeds = l + 1 < self.L and self.chained[l + 1]
+            self.dy[l] = self.dx[l + 1] if feeds else torch.zeros(self.shapes[l][0], _align(self.shapes[l][2]), **f16)
+        need = 0
+        for m, k, n in self.shapes:
+            for op in (mp.MP_OP_FWD, mp.MP_OP_DGRAD, mp.MP_OP_WGRAD):
+                need = max(need, mp.mp_gemm_workspace_bytes(m, k, n, op))
+        self.workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=self.device)
+
+    # ---- data movement (no arithmetic) ----
+    def load_weights(self, l: int, w32: torch.Tensor, w16: torch.Tensor):
+        """Copies an FP32 master [K,N] and its FP16 working copy into the stack."""
+        n = self.shapes[l][2]
+        self.w32[l][:, :n].copy_(w32)
+        self.w16[l][:, :n].copy_(w16)
+
+    def X(self, l): return self.x[l][:, :self.shapes[l][1]]
+    def Y(self, l): return self.y[l][:, :self.shapes[l][2]]
+    def dY(self, l): return self.dy[l][:, :self.shapes[l][2]]
+    def dX(self, l): return self.dx[l][:, :self.shapes[l][1]]
+    def dW(self, l): return self.dw[l][:, :self.shapes[l][2]]
+    def W16(self, l): return self.w16[l][:, :self.shapes[l][2]]
+    def W32(self, l): return self.w32[l][:, :self.shapes[l][2]]
+
+    def feeds_next(self, l):
+        return l + 1 < self.L and self.chained[l + 1]
+
+    # ---- the step ----
+    def step(self, xs, gs):
+        """xs[l]: FP16 [M,K] CUDA tensor (row pitch a multiple of 8) for a layer that is not
+        chained; gs[l]: contiguous FP32 [M,N] CUDA tensor, the unscaled gradient entering a layer
+        whose output feeds no chained layer."""
+        for l in range(self.L):
+            if not self.chained[l]:
+                self.x[l] = xs[l]
+            mp.mp_linear_fwd(self.x[l][:, :self.shapes[l][1]], self.W16(l), self.Y(l), self.workspace)
+        for l in range(self.L - 1, -1, -1):
+            if not self.feeds_next(l):
+                n = self.shapes[l][2]
+                if self.dy[l].shape[1] == n:
+                    mp.mp_scale_upstream(gs[l], self.dy[l], self.state)
+                else:   # padded rows: scale into a dense buffer, then place (copy only)
+                    tmp = torch.empty(self.shapes[l][0], n, dtype=torch.float16, device=self.device)
+                    mp.mp_scale_upstream(gs[l], tmp, self.state)
+                    self.dy[l][:, :n].copy_(tmp)
+            X = self.x[l][:, :self.shapes[l][1]]
+            mp.mp_linear_bwd_wgrad(X, self.dY(l), self.dW(l), self.state, self.workspace)
+            mp.mp_linear_bwd_dgrad(self.dY(l), self.W16(l), self.dX(l), self.workspace)
+        mp.mp_master_update(self.plan, self.state, self.opt, 0)
+        mp.mp_loss_scale_update(self.state)
+
+    def close(self):
+        self.plan.close()
+        self.state.close()

@@ -17,3 +17,14 @@ def orc():
     from oracle import mp_oracle
     mp_oracle.build()
     return mp_oracle
+
+
+@pytest.fixture(scope="session")
+def mp():
+    """The Python binding of the CUDA library; GPU tests only."""
+    import torch
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_1805_10387_b200 import mp as binding
+    binding.lib()
+    return binding

@@ -1,0 +1,134 @@
+"""The whole step on the GPU (five C-ABI calls per layer stack) against the oracle's step."""
+import numpy as np
+import pytest
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+from paper_1805_10387_b200 import synth  # noqa: E402
+
+
+def _bits(t):
+    return t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+def _f(bits):
+    return bits.view(np.float16).astype(np.float64)
+
+
+def _pad_dev(bits):
+    r, c = bits.shape
+    buf = torch.zeros(r, (c + 7) // 8 * 8, dtype=torch.float16, device="cuda")
+    buf[:, :c] = torch.from_numpy(bits.view(np.float16)).cuda()
+    return buf
+
+
+def build_both(orc, cfg):
+    from paper_1805_10387_b200.stack import LinearStack
+    L = len(cfg.shapes)
+    chained = [cfg.chained(l) for l in range(L)]
+    gpu = LinearStack(cfg.shapes, chained, optimizer=cfg.optimizer, lr=cfg.lr, beta1=cfg.beta1,
+                      beta2=cfg.beta2, eps=cfg.eps, momentum=cfg.momentum,
+                      init_scale=cfg.init_scale, growth_interval=cfg.growth_interval)
+    layers = []
+    for l in range(L):
+        w = synth.weights(cfg, l)
+        ly = orc.make_layer(w, cfg.optimizer, chained[l])
+        layers.append(ly)
+        gpu.load_weights(l, torch.from_numpy(w).cuda(),
+                         torch.from_numpy(synth.fp16_bits(w).view(np.float16).reshape(w.shape)).cuda())
+        assert (synth.fp16_bits(w).reshape(w.shape) == ly.w16).all()
+    sc = orc.Scaler(cfg.init_scale, cfg.growth_interval)
+    opt = orc.Optim(kind=cfg.optimizer, lr=cfg.lr, beta1=cfg.beta1, beta2=cfg.beta2, eps=cfg.eps,
+                    momentum=cfg.momentum)
+    return gpu, layers, sc, opt
+
+
+def close_enough(got_bits, want_bits, what):
+    """GEMM outputs: max relative error 1e-2 over elements that are not tiny; non-finite
+    patterns must agree in kind."""
+    g, w = _f(got_bits), _f(want_bits)
+    fin = np.isfinite(w) & np.isfinite(g)
+    assert (np.isfinite(w) == np.isfinite(g)).mean() > 0.9999, what
+    rms = np.sqrt((w[fin] ** 2).mean()) if fin.any() else 0.0
+    big = fin & (np.abs(w) >= 1e-3 * rms) & (np.abs(w) > 2.0 ** -14)
+    if big.any():
+        rel = np.abs(g[big] - w[big]) / np.abs(w[big])
+        assert rel.max() <= 1e-2, (what, rel.max())
+
+
+def run_config(orc, mp, cfg, steps, forced_check=True):
+    gpu, layers, sc, opt = build_both(orc, cfg)
+    L = len(cfg.shapes)
+    import copy
+    forced = None
+    records = []
+    for step in range(steps):
+        xs = [None if cfg.chained(l) else synth.activations(cfg, l, step) for l in range(L)]
+        gs = [None if cfg.feeds_next(l) else synth.upstream(cfg, l, step) for l in range(L)]
+        dxs = [None if x is None else _pad_dev(x) for x in xs]
+        dgs = [None if g is None else torch.from_numpy(g).cuda() for g in gs]
+        # state of the GPU before the step, for the teacher-forced update check
+        pre = [(gpu.W32(l).cpu().numpy().copy(), gpu.m[l][:, :cfg.shapes[l][2]].cpu().numpy().copy(),
+                None if gpu.v is None else gpu.v[l][:, :cfg.shapes[l][2]].cpu().numpy().copy())
+               for l in range(L)]
+        t_pre = gpu.state.read().t
+        gpu.step(dxs, dgs)
+        rec = orc.train_step(layers, xs, gs, sc, opt)
+        torch.cuda.synchronize()
+        assert mp.mp_gemm_device_status() == 0
+        h = gpu.state.read()
+        log = gpu.state.read_log(1)[0]
+        # flags, skip decision and scale: bit exact
+        assert log.found_inf == rec.found_inf, step
+        assert (log.scale_before, log.scale_after) == (rec.S_before, rec.S_after), step
+        assert (h.t, h.good_steps, h.skipped) == (sc.t, sc.good, sc.skipped)
+        records.append(rec)
+        for l in range(L):
+            n = cfg.shapes[l][2]
+            close_enough(_bits(gpu.Y(l)), layers[l].Y, f"Y{l} step {step}")
+            close_enough(_bits(gpu.dX(l)), layers[l].dX, f"dX{l} step {step}")
+            close_enough(_bits(gpu.dW(l)), layers[l].dW, f"dW{l} step {step}")
+            w_gpu = gpu.W32(l).cpu().numpy()
+            if rec.found_inf:                       # skipped: bitwise unchanged
+                assert (w_gpu.view(np.uint32) == pre[l][0].view(np.uint32)).all()
+                assert h.t == t_pre
+            else:
+                # free-running oracle: gradients may differ by an FP16 rounding
+                assert np.abs(w_gpu - layers[l].w32).max() <= 20 * cfg.lr * 2.0 ** -9 + 1e-7
+                if forced_check:
+                    # the oracle's update fed with the GPU's own FP16 gradient and prior state
+                    w, m, v = pre[l]
+                    w16 = np.zeros(w.shape, np.uint16)
+                    g16 = np.ascontiguousarray(_bits(gpu.dW(l)))
+                    if cfg.optimizer == "adam":
+                        orc.adam_update(g16, w, m, v, w16, rec.S_before, cfg.lr, cfg.beta1, cfg.beta2,
+                                        cfg.eps, t_pre + 1)
+                    else:
+                        orc.momentum_update(g16, w, m, w16, rec.S_before, cfg.lr, cfg.momentum)
+                    assert (np.abs(w_gpu - w) <= 1e-6 * np.maximum(np.abs(w), cfg.lr)).all()
+                    assert (_bits(gpu.W16(l)) == orc.f2h(w_gpu)).all()
+    gpu.close()
+    return records
+
+
+def test_c1_ten_steps_with_injected_inf(orc, mp):
+    cfg = synth.config("c1")
+    recs = run_config(orc, mp, cfg, cfg.steps)
+    assert [r.found_inf for r in recs] == [0, 0, 0, 0, 1, 0, 0, 0, 0, 0]
+    assert [np.log2(r.S_after) for r in recs] == [16, 16, 16, 17, 16, 16, 16, 16, 17, 17]
+
+
+@pytest.mark.parametrize("name,rows,shapes", [
+    ("c2", 320, [(320, 264, 520)] * 3),                               # unchained gate-GEMM layers
+    ("c3", 384, [(384, 136, 520), (384, 520, 136), (384, 136, 136), (384, 136, 136)]),  # FFN pair chained
+    ("c4", 512, [(512, 200, 200)] * 2 + [(512, 200, 29)]),            # chained, momentum, narrow top
+])
+def test_scaled_down_workloads(orc, mp, name, rows, shapes):
+    """The c2-c4 recipes with widths shrunk so that the oracle finishes in seconds: same value
+    distributions, optimizer and scaler; several tiles and ragged tails per product."""
+    cfg = synth.config(name)
+    cfg.shapes = shapes
+    cfg.growth_interval = 2
+    recs = run_config(orc, mp, cfg, 4)
+    assert len(recs) == 4
