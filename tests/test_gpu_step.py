@@ -44,34 +44,54 @@ def build_both(orc, cfg):
     return gpu, layers, sc, opt
 
 
-def close_enough(got_bits, want_bits, what):
-    """GEMM outputs: max relative error 1e-2 over elements that are not tiny; non-finite
-    patterns must agree in kind."""
+def drift_ok(got_bits, want_bits, what):
+    """Free-running comparison: the two sides see inputs that may already differ by an FP16
+    rounding (chained layers, updated weights), so the error is measured against the size of
+    the tensor, not of each element."""
     g, w = _f(got_bits), _f(want_bits)
     fin = np.isfinite(w) & np.isfinite(g)
     assert (np.isfinite(w) == np.isfinite(g)).mean() > 0.9999, what
-    rms = np.sqrt((w[fin] ** 2).mean()) if fin.any() else 0.0
-    big = fin & (np.abs(w) >= 1e-3 * rms) & (np.abs(w) > 2.0 ** -14)
-    if big.any():
-        rel = np.abs(g[big] - w[big]) / np.abs(w[big])
-        assert rel.max() <= 1e-2, (what, rel.max())
+    if fin.any():
+        rms = np.sqrt((w[fin] ** 2).mean())
+        err = np.abs(g[fin] - w[fin])
+        assert (err <= 1e-2 * np.abs(w[fin]) + 2e-2 * rms + 2.0 ** -24).all(), (what, err.max(), rms)
 
 
-def run_config(orc, mp, cfg, steps, forced_check=True):
+def forced_ok(orc, op, A_bits, B_bits, got_bits, what):
+    """The oracle's product of the very operands the GPU kernel read: bounded by one FP16
+    rounding plus FP32 summation-order error, and max relative error 1e-2 where not tiny."""
+    A = np.ascontiguousarray(A_bits); B = np.ascontiguousarray(B_bits)
+    want = {"fwd": orc.linear_fwd, "dgrad": orc.linear_bwd_dgrad, "wgrad": orc.linear_bwd_wgrad}[op](A, B)
+    ex, ab = orc.linear_exact(op, A, B)
+    red = {"fwd": A.shape[1], "dgrad": A.shape[1], "wgrad": A.shape[0]}[op]
+    g, w = _f(got_bits), _f(want)
+    fin = np.isfinite(ex) & (np.abs(ex) < 65000.0)
+    tol = 2.0 ** -10 * np.abs(ex) + red * 2.0 ** -24 * ab + 2.0 ** -24
+    assert (np.abs(g - ex)[fin] <= tol[fin]).all(), what
+    inf_w = ~np.isfinite(w)
+    assert (np.isfinite(g) == np.isfinite(w))[~fin | inf_w].mean() > 0.99 if (~fin | inf_w).any() else True
+    both = np.isfinite(w) & np.isfinite(g)
+    if both.any():
+        rms = np.sqrt((w[both] ** 2).mean())
+        big = both & (np.abs(w) >= 1e-3 * rms) & (np.abs(w) > 2.0 ** -14)
+        if big.any():
+            assert (np.abs(g[big] - w[big]) / np.abs(w[big])).max() <= 1e-2, what
+
+
+def run_config(orc, mp, cfg, steps):
     gpu, layers, sc, opt = build_both(orc, cfg)
     L = len(cfg.shapes)
-    import copy
-    forced = None
     records = []
     for step in range(steps):
         xs = [None if cfg.chained(l) else synth.activations(cfg, l, step) for l in range(L)]
         gs = [None if cfg.feeds_next(l) else synth.upstream(cfg, l, step) for l in range(L)]
         dxs = [None if x is None else _pad_dev(x) for x in xs]
         dgs = [None if g is None else torch.from_numpy(g).cuda() for g in gs]
-        # state of the GPU before the step, for the teacher-forced update check
+        # state of the GPU before the step, for the checks that reuse the GPU's own operands
         pre = [(gpu.W32(l).cpu().numpy().copy(), gpu.m[l][:, :cfg.shapes[l][2]].cpu().numpy().copy(),
                 None if gpu.v is None else gpu.v[l][:, :cfg.shapes[l][2]].cpu().numpy().copy())
                for l in range(L)]
+        w16_pre = [_bits(gpu.W16(l)) for l in range(L)]
         t_pre = gpu.state.read().t
         gpu.step(dxs, dgs)
         rec = orc.train_step(layers, xs, gs, sc, opt)
@@ -85,29 +105,38 @@ def run_config(orc, mp, cfg, steps, forced_check=True):
         assert (h.t, h.good_steps, h.skipped) == (sc.t, sc.good, sc.skipped)
         records.append(rec)
         for l in range(L):
-            n = cfg.shapes[l][2]
-            close_enough(_bits(gpu.Y(l)), layers[l].Y, f"Y{l} step {step}")
-            close_enough(_bits(gpu.dX(l)), layers[l].dX, f"dX{l} step {step}")
-            close_enough(_bits(gpu.dW(l)), layers[l].dW, f"dW{l} step {step}")
+            Xg, Yg, dYg = _bits(gpu.X(l)), _bits(gpu.Y(l)), _bits(gpu.dY(l))
+            dXg, dWg = _bits(gpu.dX(l)), _bits(gpu.dW(l))
+            forced_ok(orc, "fwd", Xg, w16_pre[l], Yg, f"Y{l} step {step}")
+            forced_ok(orc, "wgrad", Xg, dYg, dWg, f"dW{l} step {step}")
+            forced_ok(orc, "dgrad", dYg, w16_pre[l], dXg, f"dX{l} step {step}")
+            if not cfg.feeds_next(l):              # upstream scaling: bitwise
+                assert (dYg == orc.scale_upstream(gs[l], rec.S_before)).all()
+            drift_ok(Yg, layers[l].Y, f"Y{l} step {step}")
+            drift_ok(dXg, layers[l].dX, f"dX{l} step {step}")
+            drift_ok(dWg, layers[l].dW, f"dW{l} step {step}")
             w_gpu = gpu.W32(l).cpu().numpy()
             if rec.found_inf:                       # skipped: bitwise unchanged
                 assert (w_gpu.view(np.uint32) == pre[l][0].view(np.uint32)).all()
+                assert (_bits(gpu.W16(l)) == w16_pre[l]).all()
                 assert h.t == t_pre
             else:
-                # free-running oracle: gradients may differ by an FP16 rounding
-                assert np.abs(w_gpu - layers[l].w32).max() <= 20 * cfg.lr * 2.0 ** -9 + 1e-7
-                if forced_check:
-                    # the oracle's update fed with the GPU's own FP16 gradient and prior state
-                    w, m, v = pre[l]
-                    w16 = np.zeros(w.shape, np.uint16)
-                    g16 = np.ascontiguousarray(_bits(gpu.dW(l)))
-                    if cfg.optimizer == "adam":
-                        orc.adam_update(g16, w, m, v, w16, rec.S_before, cfg.lr, cfg.beta1, cfg.beta2,
-                                        cfg.eps, t_pre + 1)
-                    else:
-                        orc.momentum_update(g16, w, m, w16, rec.S_before, cfg.lr, cfg.momentum)
-                    assert (np.abs(w_gpu - w) <= 1e-6 * np.maximum(np.abs(w), cfg.lr)).all()
-                    assert (_bits(gpu.W16(l)) == orc.f2h(w_gpu)).all()
+                # free-running oracle: its gradients may differ by an FP16 rounding, and Adam
+                # turns a sign flip of a near-zero gradient into a full step of size lr
+                diff = np.abs(w_gpu - layers[l].w32)
+                assert diff.max() <= 2.5 * cfg.lr * (h.t if cfg.optimizer == "adam" else 1) + 1e-7
+                assert np.median(diff) <= 1e-6
+                # the oracle's update fed with the GPU's own FP16 gradient and prior state
+                w, m, v = pre[l]
+                w16 = np.zeros(w.shape, np.uint16)
+                g16 = np.ascontiguousarray(dWg)
+                if cfg.optimizer == "adam":
+                    orc.adam_update(g16, w, m, v, w16, rec.S_before, cfg.lr, cfg.beta1, cfg.beta2,
+                                    cfg.eps, t_pre + 1)
+                else:
+                    orc.momentum_update(g16, w, m, w16, rec.S_before, cfg.lr, cfg.momentum)
+                assert (np.abs(w_gpu - w) <= 1e-6 * np.maximum(np.abs(w), cfg.lr)).all()
+                assert (_bits(gpu.W16(l)) == orc.f2h(w_gpu)).all()
     gpu.close()
     return records
 
