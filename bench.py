@@ -1,0 +1,331 @@
+#!/usr/bin/env python
+"""Benchmark of the mixed-precision training step of a linear-layer stack on B200.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2|c3|c4] [--impl reference]
+
+One step = forward, weight-gradient and data-gradient products of every layer (FP16 operands,
+FP32 accumulation), upstream scaling, the fused unscale / inspect / FP32-master optimizer /
+FP16 recast update and the loss-scale state machine, on one batch of seeded synthetic input.
+Prints ONE JSON line.  `value` is the whole job's GEMM throughput over the step time (inputs
+resident in HBM); `e2e` is the same with pinned host inputs copied in and the loss-scale state
+read back every step; `roofline` is for the dominant kernel (the tcgen05 GEMM), timed with CUDA
+events around each launch inside the timed region; `update` gives the fused update's GB/s.
+`--impl reference` times the CPU oracle (the slow, plain restatement of the method) instead.
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "MP train step: GEMM TFLOP/s and master-update GB/s, % of B200 peak"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+# DRAM bytes per launch of the GEMM kernel from one ncu capture (dram__bytes_read.sum +
+# dram__bytes_write.sum), keyed by workload, valid only for the kernel source it was taken on.
+NCU_TRAFFIC = {"sha": "", "bytes_per_launch": {}}
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {k: float(p[k]) for k in FALLBACK_PEAKS}, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+def kernel_sha():
+    h = hashlib.sha256()
+    for f in ("gemm.cu", "ptx.cuh"):
+        h.update(open(os.path.join(ROOT, "paper_1805_10387_b200", "csrc", f), "rb").read())
+    return h.hexdigest()[:16]
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.rows, self.proc, self.index = [], None, index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        self.thread.join(timeout=2)
+        sm = sorted(float(r[0]) for r in self.rows if r and r[0].replace(".", "").isdigit())
+        mx = [float(r[1]) for r in self.rows if len(r) > 1 and r[1].replace(".", "").isdigit()]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for i, n in enumerate(names) if any(len(r) > 3 + i and r[3 + i] == "Active" for r in self.rows)]
+        pw = [float(r[2]) for r in self.rows if len(r) > 2 and r[2].replace(".", "").isdigit()]
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": mx[0] if mx else None,
+                "reasons": reasons, "samples": len(sm), "power_w_max": max(pw) if pw else None}
+
+
+# ------------------------------------------------------------------ reference arm (CPU oracle)
+def oracle_sample_step(orc, synth, cfg, rows, upd_params, data=None):
+    """One bounded sample of the workload on the CPU oracle: the three products of layer 0 on
+    its first `rows` rows and the optimizer update of `upd_params` parameters.  Returns
+    (seconds, gemm_flops, update_bytes, data)."""
+    import numpy as np
+    M, K, N = cfg.shapes[0]
+    if data is None:
+        w = synth.weights(cfg, 0)
+        X = np.ascontiguousarray(synth.activations(cfg, 0, 0)[:rows])
+        g = np.ascontiguousarray(synth.upstream(cfg, 0, 0)[:rows])
+        W16 = synth.fp16_bits(w).reshape(K, N)
+        n = min(upd_params, K * N)
+        st = dict(w32=w.reshape(-1)[:n].copy(), m=np.zeros(n, np.float32), v=np.zeros(n, np.float32),
+                  w16=np.zeros(n, np.uint16))
+        data = (X, g, W16, st)
+    X, g, W16, st = data
+    S = 2.0 ** 10
+    t0 = time.perf_counter()
+    orc.linear_fwd(X, W16)
+    dY = orc.scale_upstream(g, S)
+    dW = orc.linear_bwd_wgrad(X, dY)
+    orc.linear_bwd_dgrad(dY, W16)
+    n = st["w32"].size
+    g16 = np.ascontiguousarray(dW.reshape(-1)[:n])
+    if not orc.found_inf(dW):
+        if cfg.optimizer == "adam":
+            orc.adam_update(g16, st["w32"], st["m"], st["v"], st["w16"], S, cfg.lr, cfg.beta1, cfg.beta2, cfg.eps, 1)
+        else:
+            orc.momentum_update(g16, st["w32"], st["m"], st["w16"], S, cfg.lr, cfg.momentum)
+    dt = time.perf_counter() - t0
+    return dt, 3 * 2 * rows * K * N, n * (28 if cfg.optimizer == "adam" else 20), data
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import mp_oracle as orc
+    from paper_1805_10387_b200 import synth
+    orc.build()
+    cfg = synth.config(args.workload)
+    rows, upd = 48, 1 << 20
+    data = None
+    for _ in range(args.warmup):
+        _, _, _, data = oracle_sample_step(orc, synth, cfg, rows, upd, data)
+    tot, flops = 0.0, 0
+    for _ in range(args.steps):
+        dt, f, _, data = oracle_sample_step(orc, synth, cfg, rows, upd, data)
+        tot += dt
+        flops += f
+    val = flops / tot / 1e12
+    cores = orc.hardware_threads()
+    sample = f"per step: fwd+wgrad+dgrad of layer 0 on its first {rows} rows + update of {upd} params"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": "TFLOP/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": tot / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f16 in / f32 accumulate",
+        "data": "synthetic", "config": {"workload": cfg.name + ": " + cfg.note},
+        "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+# ------------------------------------------------------------------ CUDA arm
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--workload", default="c2", choices=["c2", "c3", "c4"])
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import numpy as np
+    import torch
+    from paper_1805_10387_b200 import mp, synth
+    from paper_1805_10387_b200.stack import LinearStack
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    mp.lib()
+
+    cfg = synth.config(args.workload)
+    L = len(cfg.shapes)
+    chained = [cfg.chained(l) for l in range(L)]
+    stack = LinearStack(cfg.shapes, chained, optimizer=cfg.optimizer, lr=cfg.lr, beta1=cfg.beta1,
+                        beta2=cfg.beta2, eps=cfg.eps, momentum=cfg.momentum, init_scale=cfg.init_scale,
+                        growth_interval=cfg.growth_interval)
+    if world > 1:      # data parallel over rows: weights replicated, FP16 weight gradients summed
+        stack.grad_sync = lambda flat: dist.all_reduce(flat)
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(1234 + cfg.seed)           # same weights on every rank
+    for l, (M, K, N) in enumerate(cfg.shapes):
+        w = torch.randn(K, N, generator=gen, device="cuda") / K ** 0.5
+        stack.load_weights(l, w, w.half())
+    gen.manual_seed(99 + rank)                 # each rank its own rows
+    xs, gs, xs_host, gs_host = [], [], [], []
+    for l, (M, K, N) in enumerate(cfg.shapes):
+        if chained[l]:
+            xs.append(None); xs_host.append(None)
+        else:
+            z = torch.randn(M, K, generator=gen, device="cuda")
+            if cfg.x_dist == "lognormal2":
+                z = torch.sign(torch.randn(M, K, generator=gen, device="cuda")) * torch.clamp(torch.exp(2 * z), max=6.0e4)
+            x = torch.zeros(M, (K + 7) // 8 * 8, dtype=torch.float16, device="cuda")
+            x[:, :K] = z.half()
+            xs.append(x)
+            xs_host.append(x[:, :K].contiguous().cpu().pin_memory())
+        if stack.feeds_next(l):
+            gs.append(None); gs_host.append(None)
+        else:
+            g = torch.randn(M, N, generator=gen, device="cuda") * cfg.grad_std
+            gs.append(g)
+            gs_host.append(g.cpu().pin_memory())
+    h2d = sum(t.numel() * t.element_size() for t in xs_host + gs_host if t is not None)
+    d2h = 56
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps):
+        """max over ranks of the device time of `steps` calls, in ms"""
+        barrier()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(steps):
+            fn()
+        b.record()
+        barrier()
+        ms = torch.tensor([a.elapsed_time(b)], device="cuda")
+        if dist is not None:
+            dist.all_reduce(ms, op=dist.ReduceOp.MAX)
+        return float(ms.item())
+
+    for _ in range(max(args.warmup, 3)):
+        stack.step(xs, gs)
+    torch.cuda.synchronize()
+    st0 = stack.state.read()
+    launches0 = mp.mp_kernel_launch_count()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    stack.events = []
+    ms_total = timed(lambda: stack.step(xs, gs), args.steps)
+    events, stack.events = stack.events, None
+    launches = mp.mp_kernel_launch_count() - launches0
+    st1 = stack.state.read()
+    # end to end: pinned host inputs in, loss-scale state out, every step
+    for _ in range(2):
+        stack.step_from_host(xs_host, gs_host)
+    ms_e2e = timed(lambda: stack.step_from_host(xs_host, gs_host), args.steps)
+    clocks = sampler.stop() if rank == 0 else None
+    assert mp.mp_gemm_device_status() == 0, "a GEMM kernel reported a device-side error"
+
+    # per-call device times from the events recorded inside the timed region
+    per = {}
+    for name, a, b in events:
+        per.setdefault(name, []).append(a.elapsed_time(b))
+    flops_step = cfg.gemm_flops()
+    ms_step = ms_total / args.steps
+    value = world * flops_step / (ms_step * 1e-3) / 1e12
+    e2e_val = world * flops_step / (ms_e2e / args.steps * 1e-3) / 1e12
+    pk, pk_src = peaks()
+    gemm_ms = sum(sum(per.get(k, [])) for k in ("fwd", "dgrad", "wgrad"))
+    gemm_calls = sum(len(per.get(k, [])) for k in ("fwd", "dgrad", "wgrad"))
+    gemm_tflops = flops_step * args.steps / (gemm_ms * 1e-3) / 1e12
+    skipped = st1.skipped - st0.skipped
+    bytes_per_param = 28 if cfg.optimizer == "adam" else 20
+    upd_ms = per.get("update", [0.0])
+    applied = [t for t in upd_ms]
+    upd_bytes = cfg.n_params() * bytes_per_param
+    # skipped steps return at once; GB/s is quoted on the applied ones only
+    applied_ms = sorted(applied)[skipped:] if skipped < len(applied) else applied
+    upd_gbs = upd_bytes / (sum(applied_ms) / len(applied_ms) * 1e-3) / 1e9
+    sha = kernel_sha()
+    traffic = NCU_TRAFFIC["bytes_per_launch"].get(args.workload) if NCU_TRAFFIC["sha"] == sha else None
+    out = {
+        "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f16 in / f32 accumulate", "data": "synthetic",
+        "config": {"workload": cfg.name + ": " + cfg.note, "layers": L, "params": cfg.n_params(),
+                   "gemm_gflop_per_step": flops_step / 1e9, "optimizer": cfg.optimizer,
+                   "parallelism": f"dp{world}" if world > 1 else "single",
+                   "cache": "per-step working set (weights, moments, activations) far exceeds the 126 MB L2"},
+        "e2e": {"value": e2e_val, "unit": "TFLOP/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "ms_per_step": ms_e2e / args.steps},
+        "gpu_launches": int(launches),
+        "skipped_steps_in_timed_region": int(skipped),
+        "loss_scale": st1.scale,
+        "roofline": {"kernel": "mp_gemm_kernel", "bound": "tensor", "achieved": gemm_tflops,
+                     "peak": pk["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                     "frac": gemm_tflops / pk["bf16_tflops_sustained"], "traffic": traffic,
+                     "peak_source": f"{pk_src} cuBLAS bf16 sustained (fp16 nominal ratio 1.0)",
+                     "frac_of_burst_peak": gemm_tflops / pk["bf16_tflops"],
+                     "frac_of_nominal_2250": gemm_tflops / 2250.0,
+                     "launches": gemm_calls, "avg_launch_ms": gemm_ms / max(gemm_calls, 1),
+                     "per_op_tflops": {k: (flops_step / 3) * args.steps / (sum(per[k]) * 1e-3) / 1e12
+                                       for k in ("fwd", "dgrad", "wgrad") if k in per}},
+        "update": {"kernel": "mp_master_update_kernel", "bound": "hbm", "achieved": upd_gbs,
+                   "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": upd_gbs / pk["hbm_gbs"],
+                   "frac_of_nominal_8000": upd_gbs / 8000.0, "bytes_per_param": bytes_per_param,
+                   "avg_launch_ms": sum(applied_ms) / len(applied_ms), "peak_source": pk_src + " copy"},
+        "clocks": clocks,
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        from oracle import mp_oracle as orc
+        orc.build()
+        rows, upd = 64, 1 << 21
+        tot, fl, data = 0.0, 0, None
+        t_budget = time.perf_counter()
+        while tot < 12.0 and time.perf_counter() - t_budget < 40.0:
+            dt, f, _, data = oracle_sample_step(orc, synth, cfg, rows, upd, data)
+            tot += dt
+            fl += f
+        out["cpu_baseline"] = {"value": fl / tot / 1e12, "unit": "TFLOP/s", "cores": orc.hardware_threads(),
+                               "kind": "oracle",
+                               "sample": f"fwd+wgrad+dgrad of layer 0 on its first {rows} rows + update of "
+                                         f"{upd} params, repeated for {tot:.1f} s"}
+    if rank == 0:
+        print(json.dumps(out))
+    stack.close()
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

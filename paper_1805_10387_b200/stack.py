@@ -94,6 +94,39 @@ class LinearStack:
     def feeds_next(self, l):
         return l + 1 < self.L and self.chained[l + 1]
 
+    # ---- optional per-call device timing (CUDA events on the launching stream) ----
+    events = None   # set to a list to collect (name, start_event, end_event)
+    grad_sync = None  # data-parallel runs: callable that all-reduces the flat FP16 gradient
+
+    def _call(self, name, fn, *args):
+        if self.events is None:
+            fn(*args)
+            return
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        fn(*args)
+        b.record()
+        self.events.append((name, a, b))
+
+    def step_from_host(self, xs_host, gs_host):
+        """The step as a caller with host data makes it: pinned host inputs are copied to the
+        device, the step runs, and the loss-scale state comes back to the host."""
+        L = self.L
+        if not hasattr(self, "_x_in"):
+            self._x_in = [None if self.chained[l] else
+                          torch.empty(self.shapes[l][0], _align(self.shapes[l][1]), dtype=torch.float16,
+                                      device=self.device) for l in range(L)]
+            self._g_in = [None if self.feeds_next(l) else
+                          torch.empty(self.shapes[l][0], self.shapes[l][2], dtype=torch.float32,
+                                      device=self.device) for l in range(L)]
+        for l in range(L):
+            if self._x_in[l] is not None:
+                self._x_in[l][:, :self.shapes[l][1]].copy_(xs_host[l], non_blocking=True)
+            if self._g_in[l] is not None:
+                self._g_in[l].copy_(gs_host[l], non_blocking=True)
+        self.step(self._x_in, self._g_in)
+        return self.state.read()
+
     # ---- the step ----
     def step(self, xs, gs):
         """xs[l]: FP16 [M,K] CUDA tensor (row pitch a multiple of 8) for a layer that is not
@@ -102,21 +135,27 @@ class LinearStack:
         for l in range(self.L):
             if not self.chained[l]:
                 self.x[l] = xs[l]
-            mp.mp_linear_fwd(self.x[l][:, :self.shapes[l][1]], self.W16(l), self.Y(l), self.workspace)
+            self._call("fwd", mp.mp_linear_fwd, self.x[l][:, :self.shapes[l][1]], self.W16(l), self.Y(l),
+                       self.workspace)
         for l in range(self.L - 1, -1, -1):
             if not self.feeds_next(l):
                 n = self.shapes[l][2]
                 if self.dy[l].shape[1] == n:
-                    mp.mp_scale_upstream(gs[l], self.dy[l], self.state)
+                    self._call("scale", mp.mp_scale_upstream, gs[l], self.dy[l], self.state)
                 else:   # padded rows: scale into a dense buffer, then place (copy only)
                     tmp = torch.empty(self.shapes[l][0], n, dtype=torch.float16, device=self.device)
                     mp.mp_scale_upstream(gs[l], tmp, self.state)
                     self.dy[l][:, :n].copy_(tmp)
             X = self.x[l][:, :self.shapes[l][1]]
-            mp.mp_linear_bwd_wgrad(X, self.dY(l), self.dW(l), self.state, self.workspace)
-            mp.mp_linear_bwd_dgrad(self.dY(l), self.W16(l), self.dX(l), self.workspace)
-        mp.mp_master_update(self.plan, self.state, self.opt, 0)
-        mp.mp_loss_scale_update(self.state)
+            self._call("wgrad", mp.mp_linear_bwd_wgrad, X, self.dY(l), self.dW(l), self.state,
+                       self.workspace)
+            self._call("dgrad", mp.mp_linear_bwd_dgrad, self.dY(l), self.W16(l), self.dX(l),
+                       self.workspace)
+        if self.grad_sync is not None:       # data parallel: sum the FP16 gradients over ranks,
+            self.grad_sync(self.dw_flat)     # then inspect the reduced gradients in the update call
+        self._call("update", mp.mp_master_update, self.plan, self.state, self.opt,
+                   0 if self.grad_sync is None else 1)
+        self._call("scaler", mp.mp_loss_scale_update, self.state)
 
     def close(self):
         self.plan.close()
