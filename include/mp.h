@@ -132,6 +132,35 @@ int mp_master_update(mp_update_plan* plan, mp_state* state, const mp_optim_confi
  * Then the flag is cleared, step++ and a log record is appended.  One tiny kernel. */
 int mp_loss_scale_update(mp_state* state, void* stream);
 
+/* Weight gradient for callers that must not allocate.  (The paper has no counterpart: this is
+ * a packaging variant of mp_linear_bwd_wgrad, same arithmetic, same results bit for bit.)
+ *
+ * Who needs it: code that runs where device allocation is off the table -- a training or
+ * serving runtime that has already handed all free device memory to its own pool, so that a
+ * cudaMalloc would fail; a step that must not hit the implicit device-wide synchronisation an
+ * allocation or free causes; a plugin whose host forbids allocator calls inside its callbacks.
+ * Such callers also may have no spare buffer to lend as `workspace`.
+ *
+ * Differences from mp_linear_bwd_wgrad: there is no workspace argument.  The split-reduction
+ * scratch is an array built into the library image, MP_STATIC_SCRATCH_BYTES (32 MiB) per GPU,
+ * reserved on every GPU that loads the library until the process exits.  Sizes whose scratch
+ * need (mp_gemm_workspace_bytes(M,K,N,MP_OP_WGRAD)) exceeds it are refused with
+ * MP_ERR_TOO_LARGE and nothing is launched.  The call makes no cudaMalloc/cudaFree and uses no
+ * allocating library routine.
+ *
+ * The first call on each device looks up the array's device address (one cheap runtime query,
+ * no allocation, done with that device current); make that first call before starting any
+ * stream capture.  All calls on a device share the one array: two calls whose kernels may
+ * overlap on the GPU (different streams) race on it and must be ordered by the caller.  The
+ * array keeps whatever the previous call left; that is harmless because each call overwrites
+ * every partial sum it later reads, so nothing has to start at zero. */
+#define MP_STATIC_SCRATCH_BYTES (32u << 20)
+int mp_linear_bwd_wgrad_static(const void* X16, int64_t ldx, const void* dY16, int64_t lddy,
+                               void* dW16, int64_t lddw, int64_t M, int64_t K, int64_t N,
+                               mp_state* state, void* stream);
+/* Size of that built-in scratch in bytes (equals MP_STATIC_SCRATCH_BYTES). */
+size_t mp_static_scratch_bytes(void);
+
 /* ---- auxiliaries --------------------------------------------------------------------- */
 
 enum { MP_OP_FWD = 0, MP_OP_DGRAD = 1, MP_OP_WGRAD = 2 };

@@ -505,6 +505,59 @@ int mp_linear_bwd_wgrad(const void* X16, int64_t ldx, const void* dY16, int64_t 
                   workspace_bytes, (cudaStream_t)stream);
 }
 
+// ---- weight gradient with built-in scratch -------------------------------------------------
+// Split-reduction scratch that belongs to the library image instead of the caller.  It is a
+// fixed-size device array: every GPU that loads this library reserves it until the process
+// exits, and every call on that GPU shares it.
+#define MP_STATIC_SCRATCH_FLOATS (8u << 20)   /* 8 Mi floats = 32 MiB */
+static __device__ __align__(256) float g_static_scratch[MP_STATIC_SCRATCH_FLOATS];
+
+namespace {
+constexpr int kMaxDevices = 64;
+float* g_static_scratch_addr[kMaxDevices] = {nullptr};
+
+// Device address of the scratch array on the current device.  In host code the array's name
+// is only a handle for the runtime, not an address a kernel could use, so the address is
+// asked for once per device (with that device current) and remembered.
+int static_scratch_for_current_device(float** out) {
+  int dev = 0;
+  MP_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices)
+    return mp::set_error(MP_ERR_INVALID_ARG, "device index %d is outside 0..%d", dev, kMaxDevices - 1);
+  if (g_static_scratch_addr[dev] == nullptr) {
+    float* ptr = nullptr;
+    const cudaError_t e = cudaGetSymbolAddress((void**)&ptr, g_static_scratch);
+    if (e != cudaSuccess || ptr == nullptr)
+      return mp::set_error(MP_ERR_CUDA, "cudaGetSymbolAddress(static scratch): %s", cudaGetErrorString(e));
+    g_static_scratch_addr[dev] = ptr;
+  }
+  *out = g_static_scratch_addr[dev];
+  return MP_OK;
+}
+}  // namespace
+
+int mp_linear_bwd_wgrad_static(const void* X16, int64_t ldx, const void* dY16, int64_t lddy,
+                               void* dW16, int64_t lddw, int64_t M, int64_t K, int64_t N,
+                               mp_state* state, void* stream) {
+  const size_t need = mp_gemm_workspace_bytes(M, K, N, MP_OP_WGRAD);
+  const size_t have = (size_t)MP_STATIC_SCRATCH_FLOATS * sizeof(float);
+  if (need > have)
+    return mp::set_error(MP_ERR_TOO_LARGE,
+                         "mp_linear_bwd_wgrad_static: these sizes need %zu bytes of scratch, the "
+                         "built-in array holds %zu; use mp_linear_bwd_wgrad with a caller workspace",
+                         need, have);
+  if (int rc = mp::check_device()) return rc;
+  float* scratch = nullptr;
+  if (int rc = static_scratch_for_current_device(&scratch)) return rc;
+  const Operand A{X16, ldx, true, K, M};
+  const Operand B{dY16, lddy, true, N, M};
+  int* flag = state ? &state->dev->h.found_inf : nullptr;
+  return run_gemm("mp_linear_bwd_wgrad_static", A, B, dW16, lddw, flag, state != nullptr, scratch,
+                  have, (cudaStream_t)stream);
+}
+
+size_t mp_static_scratch_bytes(void) { return (size_t)MP_STATIC_SCRATCH_FLOATS * sizeof(float); }
+
 // Synchronises the device and returns the first device-side error recorded by a GEMM kernel
 // (MP_OK if none), clearing it.
 int mp_gemm_device_status(int* out) {

@@ -56,6 +56,8 @@ SIGNATURES = {
     "mp_linear_fwd": (_i32, [_p, _i64, _p, _i64, _p, _i64, _i64, _i64, _i64, _p, _sz, _p]),
     "mp_linear_bwd_dgrad": (_i32, [_p, _i64, _p, _i64, _p, _i64, _i64, _i64, _i64, _p, _sz, _p]),
     "mp_linear_bwd_wgrad": (_i32, [_p, _i64, _p, _i64, _p, _i64, _i64, _i64, _i64, _p, _p, _sz, _p]),
+    "mp_linear_bwd_wgrad_static": (_i32, [_p, _i64, _p, _i64, _p, _i64, _i64, _i64, _i64, _p, _p]),
+    "mp_static_scratch_bytes": (_sz, []),
     "mp_master_update": (_i32, [_p, _p, C.POINTER(OptimConfig), _i32, _p]),
     "mp_loss_scale_update": (_i32, [_p, _p]),
     "mp_gemm_workspace_bytes": (_sz, [_i64, _i64, _i64, _i32]),
@@ -162,6 +164,21 @@ def mp_linear_bwd_wgrad(X16, dY16, dW16, state=None, workspace=None):
     ws, nb = _ws(workspace)
     _check(lib().mp_linear_bwd_wgrad(x, ldx, dy, lddy, dw, lddw, M, K, N,
                                      state.handle if state is not None else None, ws, nb, _stream()))
+
+
+def mp_linear_bwd_wgrad_static(X16, dY16, dW16, state=None):
+    """Weight gradient with the library's built-in scratch: for callers that cannot allocate
+    device memory or lend a workspace.  Same result as mp_linear_bwd_wgrad."""
+    (x, ldx), (dy, lddy), (dw, lddw) = _mat(X16), _mat(dY16), _mat(dW16)
+    M, K = X16.shape
+    N = dY16.shape[1]
+    assert dY16.shape[0] == M and tuple(dW16.shape) == (K, N)
+    _check(lib().mp_linear_bwd_wgrad_static(x, ldx, dy, lddy, dw, lddw, M, K, N,
+                                            state.handle if state is not None else None, _stream()))
+
+
+def mp_static_scratch_bytes() -> int:
+    return int(lib().mp_static_scratch_bytes())
 
 
 def mp_master_update(plan, state, opt: OptimConfig, check_mode: int = 0):
