@@ -188,7 +188,8 @@ def main():
                         beta2=cfg.beta2, eps=cfg.eps, momentum=cfg.momentum, init_scale=cfg.init_scale,
                         growth_interval=cfg.growth_interval)
     if world > 1:      # data parallel over rows: weights replicated, FP16 weight gradients summed
-        stack.grad_sync = lambda flat: dist.all_reduce(flat)
+        from paper_1805_10387_b200 import dp
+        stack.grad_sync = dp.allreduce_gradients
     gen = torch.Generator(device="cuda")
     gen.manual_seed(1234 + cfg.seed)           # same weights on every rank
     for l, (M, K, N) in enumerate(cfg.shapes):
