@@ -67,9 +67,72 @@ __device__ __forceinline__ uint32_t pair_nonfinite(uint32_t w) {
   return __vcmpeq2(w & 0x7C007C00u, 0x7C007C00u);
 }
 
-__device__ __forceinline__ void report_timeout(Barriers* bars) {
+template <class B>
+__device__ __forceinline__ void report_timeout(B* bars) {
   bars->abort = 1;
   atomicCAS(&g_gemm_status, 0, (int)MP_ERR_TIMEOUT);
+}
+
+// Epilogue of one 128 x 256 accumulator for one warp: this thread owns output row `row`
+// (TMEM lane) and walks the columns in chunks of 32.  tmem_acc is the TMEM address of the
+// accumulator's first column in this warp's lane quarter.  Returns nonzero if an inf or NaN
+// was stored as FP16.
+__device__ __forceinline__ uint32_t epilogue_tile(const GemmParams& p, uint32_t tmem_acc, int row,
+                                                  int n0, int split) {
+  const bool row_ok = row < p.Mo;
+  uint32_t bad = 0;
+#pragma unroll 1
+  for (int c = 0; c < BN / 32; ++c) {
+    const int col0 = n0 + c * 32;
+    if (col0 >= p.No) break;                    // warp-uniform
+    uint32_t r[32];
+    ptx::tmem_ld_32x32(tmem_acc + c * 32, r);
+    ptx::tmem_ld_wait();
+    if (p.out_mode == OUT_PARTIAL) {
+      if (row_ok) {
+        float* dst = p.ws + ((int64_t)split * p.Mo + row) * p.ws_ld + col0;
+        if (col0 + 32 <= p.No) {
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            *reinterpret_cast<uint4*>(dst + 4 * j) =
+                make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
+        } else {
+#pragma unroll
+          for (int j = 0; j < 32; ++j)
+            if (col0 + j < p.No) dst[j] = __uint_as_float(r[j]);
+        }
+      }
+    } else {
+      uint32_t h[16];
+#pragma unroll
+      for (int j = 0; j < 16; ++j) {
+        const __half2 v = __floats2half2_rn(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1]));
+        h[j] = *reinterpret_cast<const uint32_t*>(&v);
+      }
+      if (row_ok) {
+        uint16_t* dst = p.out + (int64_t)row * p.ldo + col0;
+        if (col0 + 32 <= p.No) {
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            *reinterpret_cast<uint4*>(dst + 8 * j) =
+                make_uint4(h[4 * j], h[4 * j + 1], h[4 * j + 2], h[4 * j + 3]);
+            bad |= pair_nonfinite(h[4 * j]) | pair_nonfinite(h[4 * j + 1]) |
+                   pair_nonfinite(h[4 * j + 2]) | pair_nonfinite(h[4 * j + 3]);
+          }
+        } else {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            if (col0 + j < p.No) {
+              const uint16_t hv = (uint16_t)((j & 1) ? (h[j >> 1] >> 16) : (h[j >> 1] & 0xFFFFu));
+              dst[j] = hv;
+              bad |= ((hv & 0x7C00u) == 0x7C00u) ? 1u : 0u;
+            }
+          }
+        }
+      }
+    }
+  }
+  return bad;
 }
 
 template <bool A_MN, bool B_MN>
@@ -211,59 +274,7 @@ mp_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       if (!ptx::mbar_wait(&bars->tmem_full[acc], acc_phase)) { ok = false; break; }
       ptx::tc_fence_after_sync();
       const int row = m0 + q * 32 + lane;
-      const bool row_ok = row < p.Mo;
-      uint32_t bad = 0;
-#pragma unroll 1
-      for (int c = 0; c < BN / 32; ++c) {
-        const int col0 = n0 + c * 32;
-        if (col0 >= p.No) break;                    // warp-uniform
-        uint32_t r[32];
-        ptx::tmem_ld_32x32(tmem_base + acc * BN + c * 32 + ((uint32_t)(q * 32) << 16), r);
-        ptx::tmem_ld_wait();
-        if (p.out_mode == OUT_PARTIAL) {
-          if (row_ok) {
-            float* dst = p.ws + ((int64_t)split * p.Mo + row) * p.ws_ld + col0;
-            if (col0 + 32 <= p.No) {
-#pragma unroll
-              for (int j = 0; j < 8; ++j)
-                *reinterpret_cast<uint4*>(dst + 4 * j) =
-                    make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
-            } else {
-#pragma unroll
-              for (int j = 0; j < 32; ++j)
-                if (col0 + j < p.No) dst[j] = __uint_as_float(r[j]);
-            }
-          }
-        } else {
-          uint32_t h[16];
-#pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            const __half2 v = __floats2half2_rn(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1]));
-            h[j] = *reinterpret_cast<const uint32_t*>(&v);
-          }
-          if (row_ok) {
-            uint16_t* dst = p.out + (int64_t)row * p.ldo + col0;
-            if (col0 + 32 <= p.No) {
-#pragma unroll
-              for (int j = 0; j < 4; ++j) {
-                *reinterpret_cast<uint4*>(dst + 8 * j) =
-                    make_uint4(h[4 * j], h[4 * j + 1], h[4 * j + 2], h[4 * j + 3]);
-                bad |= pair_nonfinite(h[4 * j]) | pair_nonfinite(h[4 * j + 1]) |
-                       pair_nonfinite(h[4 * j + 2]) | pair_nonfinite(h[4 * j + 3]);
-              }
-            } else {
-#pragma unroll
-              for (int j = 0; j < 32; ++j) {
-                if (col0 + j < p.No) {
-                  const uint16_t hv = (uint16_t)((j & 1) ? (h[j >> 1] >> 16) : (h[j >> 1] & 0xFFFFu));
-                  dst[j] = hv;
-                  bad |= ((hv & 0x7C00u) == 0x7C00u) ? 1u : 0u;
-                }
-              }
-            }
-          }
-        }
-      }
+      const uint32_t bad = epilogue_tile(p, tmem_base + acc * BN + ((uint32_t)(q * 32) << 16), row, n0, split);
       if (p.out_mode == OUT_F16_FLAG && p.flag != nullptr) {
         if (__any_sync(0xFFFFFFFFu, bad != 0) && lane == 0) atomicOr(p.flag, 1);
       }
@@ -279,6 +290,196 @@ mp_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   if (warp == 1) {
     ptx::tc_fence_after_sync();
     ptx::tmem_dealloc(tmem_base, TMEM_COLS);
+  }
+}
+
+// ------------------------------------------------------------------ CTA-pair kernel
+// Same pipeline on a cluster of two CTAs (two SMs) that share one 256 x 256 output tile through
+// tcgen05.mma.cta_group::2: CTA r of the pair loads rows [128 r, 128 r + 128) of the A tile and
+// columns [128 r, 128 r + 128) of the B tile into its own shared memory (plain TMA loads, no
+// multicast), the leader CTA issues every MMA, and each CTA's tensor memory receives the 128
+// output rows it loaded A for.  Per SM that halves the B bytes read from shared memory per
+// flop and shrinks a stage to 32 KiB, so six stages fit.
+constexpr int STAGES2 = 6;
+constexpr int HALF_BYTES = 128 * BK * 2;            // 16 KiB: half a tile of A or of B
+constexpr int STAGE2_BYTES = 2 * HALF_BYTES;
+constexpr int SMEM2_BYTES = STAGES2 * STAGE2_BYTES + 1024 + 256;
+
+struct Barriers2 {
+  uint64_t full[STAGES2];     // used in the leader: both CTAs' loads of a stage have landed
+  uint64_t empty[STAGES2];    // in each CTA: the MMAs that read the stage are done
+  uint64_t tmem_full[2];      // in each CTA: accumulator ready for the epilogue
+  uint64_t tmem_empty[2];     // used in the leader: both CTAs' epilogues have drained it
+  uint32_t tmem_base;
+  volatile uint32_t abort;
+};
+
+template <bool A_MN, bool B_MN>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1)
+mp_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a,
+                    const __grid_constant__ CUtensorMap map_b, const GemmParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
+                                             ~static_cast<uintptr_t>(1023));
+  Barriers2* bars = reinterpret_cast<Barriers2*>(smem + STAGES2 * STAGE2_BYTES);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = ptx::cluster_ctarank();
+  const bool leader = rank == 0;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES2; ++s) {
+      ptx::mbar_init(&bars->full[s], 1);            // the leader's arrive; bytes of both CTAs
+      ptx::mbar_init(&bars->empty[s], 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      ptx::mbar_init(&bars->tmem_full[a], 1);
+      ptx::mbar_init(&bars->tmem_empty[a], 8);      // 4 epilogue warps in each CTA
+    }
+    bars->abort = 0;
+    ptx::fence_mbar_init();
+    ptx::prefetch_tensormap(&map_a);
+    ptx::prefetch_tensormap(&map_b);
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc_pair(&bars->tmem_base, TMEM_COLS);
+    ptx::tmem_relinquish_pair();
+  }
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  ptx::cluster_sync();                              // both CTAs' barriers exist before any remote arrive
+  ptx::tc_fence_after_sync();
+  const uint32_t tmem_base = bars->tmem_base;
+
+  const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
+  const int total_work = p.m_tiles * p.n_tiles * p.splits;   // m_tiles counts 256-row tiles here
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer (both CTAs)
+    int stage = 0;
+    uint32_t phase = 0;
+    int issued = 0;
+    bool ok = true;
+    for (int w = pair; w < total_work && ok; w += npairs) {
+      const int split = w % p.splits, tile = w / p.splits;
+      const int m0 = (tile / p.n_tiles) * 256 + 128 * (int)rank;
+      const int n0 = (tile % p.n_tiles) * BN + 128 * (int)rank;
+      const int kb0 = (int)((int64_t)split * p.num_kb / p.splits);
+      const int kb1 = (int)((int64_t)(split + 1) * p.num_kb / p.splits);
+      for (int kb = kb0; kb < kb1; ++kb) {
+        if (!ptx::mbar_wait(&bars->empty[stage], phase ^ 1)) { ok = false; break; }
+        if (lane == 0) {
+          uint8_t* sA = smem + stage * STAGE2_BYTES;
+          uint8_t* sB = sA + HALF_BYTES;
+          const uint32_t full = ptx::map_to_cta(ptx::smem_u32(&bars->full[stage]), 0);
+          // Only the leader arrives, expecting both CTAs' bytes.  The peer's bytes can reach the
+          // barrier before this arrive (the count of bytes still to come just goes negative
+          // for a moment); they cannot reach it before the previous phase has completed,
+          // because the peer refills a stage only after the MMAs that read it are done.
+          if (leader) ptx::mbar_arrive_expect_tx(&bars->full[stage], 2 * STAGE2_BYTES);
+          const int k = kb * BK;
+          if (A_MN) {
+            ptx::tma_load_2d_pair(sA, &map_a, full, m0, k);
+            ptx::tma_load_2d_pair(sA + CHUNK_BYTES, &map_a, full, m0 + 64, k);
+          } else {
+            ptx::tma_load_2d_pair(sA, &map_a, full, k, m0);
+          }
+          if (B_MN) {
+            ptx::tma_load_2d_pair(sB, &map_b, full, n0, k);
+            ptx::tma_load_2d_pair(sB + CHUNK_BYTES, &map_b, full, n0 + 64, k);
+          } else {
+            ptx::tma_load_2d_pair(sB, &map_b, full, k, n0);
+          }
+        }
+        __syncwarp();
+        ++issued;
+        if (++stage == STAGES2) { stage = 0; phase ^= 1; }
+      }
+    }
+    if (!ok) report_timeout(bars);
+    if (leader && (!ok || bars->abort)) {
+      // Leaving early: the leader's "full" barriers count both CTAs' bytes, so waiting on
+      // them (bounded) covers every load still in flight into either CTA; the peer cannot
+      // exit before the cluster barrier below.
+      const int pending = issued < STAGES2 ? issued : STAGES2;
+      for (int i = 0; i < pending; ++i) {
+        if (--stage < 0) { stage = STAGES2 - 1; phase ^= 1; }
+        ptx::mbar_wait(&bars->full[stage], phase);
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer (leader CTA only)
+    if (leader) {
+      constexpr uint32_t idesc = ptx::idesc_f16_f32(256, BN, A_MN, B_MN);
+      int stage = 0;
+      uint32_t phase = 0;
+      int iter = 0;
+      bool ok = true;
+      for (int w = pair; w < total_work && ok; w += npairs, ++iter) {
+        const int split = w % p.splits;
+        const int kb0 = (int)((int64_t)split * p.num_kb / p.splits);
+        const int kb1 = (int)((int64_t)(split + 1) * p.num_kb / p.splits);
+        const int acc = iter & 1;
+        const uint32_t acc_phase = (iter >> 1) & 1;
+        if (!ptx::mbar_wait(&bars->tmem_empty[acc], acc_phase ^ 1)) { ok = false; break; }
+        ptx::tc_fence_after_sync();
+        const uint32_t d_tmem = tmem_base + acc * BN;
+        for (int kb = kb0; kb < kb1; ++kb) {
+          if (!ptx::mbar_wait(&bars->full[stage], phase)) { ok = false; break; }
+          ptx::tc_fence_after_sync();
+          if (lane == 0) {
+            const uint32_t sA = ptx::smem_u32(smem + stage * STAGE2_BYTES);
+            const uint32_t sB = sA + HALF_BYTES;
+#pragma unroll
+            for (int kk = 0; kk < BK / UMMA_K; ++kk) {
+              const uint64_t da = A_MN ? ptx::smem_desc_sw128(sA + kk * 2048, CHUNK_BYTES, 1024)
+                                       : ptx::smem_desc_sw128(sA + kk * 32, 16, 1024);
+              const uint64_t db = B_MN ? ptx::smem_desc_sw128(sB + kk * 2048, CHUNK_BYTES, 1024)
+                                       : ptx::smem_desc_sw128(sB + kk * 32, 16, 1024);
+              ptx::mma_f16_ss_pair(d_tmem, da, db, idesc, (kb > kb0 || kk > 0) ? 1u : 0u);
+            }
+            ptx::mma_commit_pair(&bars->empty[stage], 3);   // frees the stage in both CTAs
+          }
+          __syncwarp();
+          if (++stage == STAGES2) { stage = 0; phase ^= 1; }
+        }
+        if (ok && lane == 0) ptx::mma_commit_pair(&bars->tmem_full[acc], 3);
+        __syncwarp();
+      }
+      if (!ok) report_timeout(bars);
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue (both CTAs)
+    const int q = warp & 3;
+    int iter = 0;
+    bool ok = true;
+    for (int w = pair; w < total_work && ok; w += npairs, ++iter) {
+      const int split = w % p.splits, tile = w / p.splits;
+      const int m0 = (tile / p.n_tiles) * 256 + 128 * (int)rank, n0 = (tile % p.n_tiles) * BN;
+      const int acc = iter & 1;
+      const uint32_t acc_phase = (iter >> 1) & 1;
+      if (!ptx::mbar_wait(&bars->tmem_full[acc], acc_phase)) { ok = false; break; }
+      ptx::tc_fence_after_sync();
+      const int row = m0 + q * 32 + lane;
+      const uint32_t bad =
+          epilogue_tile(p, tmem_base + acc * BN + ((uint32_t)(q * 32) << 16), row, n0, split);
+      if (p.out_mode == OUT_F16_FLAG && p.flag != nullptr) {
+        if (__any_sync(0xFFFFFFFFu, bad != 0) && lane == 0) atomicOr(p.flag, 1);
+      }
+      ptx::tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0)
+        ptx::mbar_arrive_cluster(ptx::map_to_cta(ptx::smem_u32(&bars->tmem_empty[acc]), 0));
+    }
+    if (!ok) report_timeout(bars);
+  }
+
+  // ---------------------------------------------------------------- teardown
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  ptx::cluster_sync();        // neither CTA's shared or tensor memory goes away under the other
+  if (warp == 1) {
+    ptx::tc_fence_after_sync();
+    ptx::tmem_dealloc_pair(tmem_base, TMEM_COLS);
   }
 }
 
@@ -354,16 +555,22 @@ int make_map(CUtensorMap* map, const void* ptr, int64_t inner, int64_t outer, in
 // Number of reduction splits: minimise a simple time model (waves of tiles on the SMs plus
 // the workspace round trip).  Depends only on the sizes, so that the workspace query and the
 // launch always agree.
+// Output tiles of more than 128 rows go to the CTA-pair kernel (256 x 256 tiles, one per SM pair).
+bool use_pair_kernel(int64_t Mo) { return Mo > 128; }
+
 int choose_splits(int64_t Mo, int64_t No, int64_t R) {
-  const int64_t tiles = ((Mo + BM - 1) / BM) * ((No + BN - 1) / BN);
+  const bool pair = use_pair_kernel(Mo);
+  const int64_t bm = pair ? 256 : BM;
+  const int64_t slots = pair ? kModelSMs / 2 : kModelSMs;
+  const int64_t tiles = ((Mo + bm - 1) / bm) * ((No + BN - 1) / BN);
   const int64_t num_kb = (R + BK - 1) / BK;
-  const double t_kb = 0.42e-6;                   // one 128x256x64 block at ~1.0e13 flop/s per SM
+  const double t_kb = 0.42e-6;                   // one 128x256x64 block per SM at ~1.0e13 flop/s
   const double bw = 4.0e12;                      // workspace traffic, bytes/s
   int best = 1;
   double best_t = 1e30;
   for (int s = 1; s <= 16 && s * 4 <= num_kb; ++s) {
     const int64_t work = tiles * s;
-    const int64_t waves = (work + kModelSMs - 1) / kModelSMs;
+    const int64_t waves = (work + slots - 1) / slots;
     double t = (double)waves * (double)((num_kb + s - 1) / s) * t_kb;
     if (s > 1) t += (double)Mo * (double)No * (8.0 * s + 2.0) / bw + 3e-6;
     if (t < best_t * 0.97) { best_t = t; best = s; }
@@ -395,6 +602,34 @@ int launch(const CUtensorMap& ma, const CUtensorMap& mb, const GemmParams& p, in
   return MP_OK;
 }
 
+template <bool A_MN, bool B_MN>
+int launch_pair(const CUtensorMap& ma, const CUtensorMap& mb, const GemmParams& p, int64_t work,
+                cudaStream_t st) {
+  static int max_pairs = 0;
+  if (max_pairs == 0) {
+    MP_CUDA_TRY(cudaFuncSetAttribute(mp_gemm_pair_kernel<A_MN, B_MN>,
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM2_BYTES));
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * kModelSMs, 1, 1);
+    cfg.blockDim = dim3(THREADS, 1, 1);
+    cfg.dynamicSmemBytes = SMEM2_BYTES;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    MP_CUDA_TRY(cudaOccupancyMaxActiveClusters(&n, mp_gemm_pair_kernel<A_MN, B_MN>, &cfg));
+    if (n < 1) return mp::set_error(MP_ERR_CUDA, "no CTA pair of the GEMM kernel fits on this device");
+    max_pairs = n;
+  }
+  const int pairs = (int)(work < max_pairs ? work : max_pairs);
+  mp_gemm_pair_kernel<A_MN, B_MN><<<2 * pairs, THREADS, SMEM2_BYTES, st>>>(ma, mb, p);
+  mp::count_launch();
+  MP_CUDA_TRY(cudaGetLastError());
+  return MP_OK;
+}
+
 int run_gemm(const char* name, const Operand& A, const Operand& B, void* out, int64_t ldo,
              int* flag, bool want_flag, void* workspace, size_t ws_bytes, cudaStream_t st) {
   const int64_t Mo = A.mn, No = B.mn, R = A.red;
@@ -416,7 +651,8 @@ int run_gemm(const char* name, const Operand& A, const Operand& B, void* out, in
 
   GemmParams p;
   p.Mo = (int)Mo; p.No = (int)No; p.R = (int)R;
-  p.m_tiles = (int)((Mo + BM - 1) / BM);
+  const bool pair = use_pair_kernel(Mo);
+  p.m_tiles = (int)(pair ? (Mo + 255) / 256 : (Mo + BM - 1) / BM);
   p.n_tiles = (int)((No + BN - 1) / BN);
   p.num_kb = (int)((R + BK - 1) / BK);
   p.splits = choose_splits(Mo, No, R);
@@ -435,7 +671,7 @@ int run_gemm(const char* name, const Operand& A, const Operand& B, void* out, in
   if (int rc = A.mn_major ? make_map(&ma, A.ptr, A.mn, A.red, A.ld, 64, BK)
                           : make_map(&ma, A.ptr, A.red, A.mn, A.ld, BK, BM)) return rc;
   if (int rc = B.mn_major ? make_map(&mb, B.ptr, B.mn, B.red, B.ld, 64, BK)
-                          : make_map(&mb, B.ptr, B.red, B.mn, B.ld, BK, BN)) return rc;
+                          : make_map(&mb, B.ptr, B.red, B.mn, B.ld, BK, pair ? 128 : BN)) return rc;
 
   int dev = 0, sms = 0;
   MP_CUDA_TRY(cudaGetDevice(&dev));
@@ -444,10 +680,17 @@ int run_gemm(const char* name, const Operand& A, const Operand& B, void* out, in
   const int grid = (int)(work < sms ? work : sms);
 
   int rc;
-  if (A.mn_major && B.mn_major) rc = launch<true, true>(ma, mb, p, grid, st);
-  else if (!A.mn_major && B.mn_major) rc = launch<false, true>(ma, mb, p, grid, st);
-  else if (!A.mn_major && !B.mn_major) rc = launch<false, false>(ma, mb, p, grid, st);
-  else rc = launch<true, false>(ma, mb, p, grid, st);
+  if (pair) {
+    if (A.mn_major && B.mn_major) rc = launch_pair<true, true>(ma, mb, p, work, st);
+    else if (!A.mn_major && B.mn_major) rc = launch_pair<false, true>(ma, mb, p, work, st);
+    else if (!A.mn_major && !B.mn_major) rc = launch_pair<false, false>(ma, mb, p, work, st);
+    else rc = launch_pair<true, false>(ma, mb, p, work, st);
+  } else {
+    if (A.mn_major && B.mn_major) rc = launch<true, true>(ma, mb, p, grid, st);
+    else if (!A.mn_major && B.mn_major) rc = launch<false, true>(ma, mb, p, grid, st);
+    else if (!A.mn_major && !B.mn_major) rc = launch<false, false>(ma, mb, p, grid, st);
+    else rc = launch<true, false>(ma, mb, p, grid, st);
+  }
   if (rc) return rc;
 
   if (p.splits > 1) {
