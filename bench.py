@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the mixed-precision training step of a linear-layer stack on B200.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2|c3|c4] [--impl reference]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2|c3|c4|c5] [--impl reference]
 
 One step = forward, weight-gradient and data-gradient products of every layer (FP16 operands,
 FP32 accumulation), upstream scaling, the fused unscale / inspect / FP32-master optimizer /
@@ -128,7 +128,7 @@ def run_reference(args):
     from oracle import mp_oracle as orc
     from paper_1805_10387_b200 import synth
     orc.build()
-    cfg = synth.config(args.workload)
+    cfg = synth.config("c2" if args.workload == "c5" else args.workload)
     rows, upd = 48, 1 << 20
     data = None
     for _ in range(args.warmup):
@@ -151,18 +151,102 @@ def run_reference(args):
     }))
 
 
+# ------------------------------------------------------------------ update-only sweep
+def run_update_sweep(args):
+    """Update-only workload: unscale / inspect / Adam / FP16 recast over 1e6 .. 1e9 parameters in
+    1 .. 500 tensors of log-uniform sizes, gradients rn16(S * N(0, 1e-3)).  Per size: GB/s on the
+    algorithmic 28 B/param for applied steps with the flag trusted (check_mode 0) and with the
+    in-call inspection (check_mode 1, 30 B/param moved), and the time of a skipped step."""
+    import torch
+    from paper_1805_10387_b200 import mp, synth
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    mp.lib()
+    pk, pk_src = peaks()
+    rows = []
+    sampler = ClockSampler(0)
+    sampler.start()
+    launches0 = mp.mp_kernel_launch_count()
+    for P, n in ((1_000_000, 1), (10_000_000, 8), (100_000_000, 64), (1_000_000_000, 500)):
+        counts = synth.tensor_sizes(P, n, 4)
+        offs, tot = [], 0
+        for c in counts:
+            offs.append(tot)
+            tot += (c + 7) // 8 * 8
+        mk = lambda dt: torch.zeros(tot, dtype=dt, device="cuda")
+        g16, w16, w32, m, v = mk(torch.float16), mk(torch.float16), mk(torch.float32), mk(torch.float32), mk(torch.float32)
+        views = lambda flat: [flat[o:o + c] for o, c in zip(offs, counts)]
+        plan = mp.UpdatePlan(views(g16), views(w32), views(m), views(v), views(w16))
+        st = mp.State(init_scale=1024.0, growth_interval=10 ** 6)
+        opt = mp.OptimConfig(mp.MP_OPT_ADAM, 1e-3, 0.9, 0.999, 1e-8, 0.9, 0.0)
+        gen = torch.Generator(device="cuda")
+        gen.manual_seed(5)
+        blk = 1 << 24
+        z = torch.randn(min(blk, tot), generator=gen, device="cuda") * (0.0316 * 1024.0)
+        for lo in range(0, tot, blk):
+            k = min(blk, tot - lo)
+            g16[lo:lo + k] = z[:k].half()
+            w32[lo:lo + k] = z[:k] * 1e-4
+        iters = max(3, min(args.steps, int(2e10 // (P * 30)) + 3))
+
+        def timed(mode, reps):
+            for _ in range(3):
+                mp.mp_master_update(plan, st, opt, mode)
+                mp.mp_loss_scale_update(st)
+            torch.cuda.synchronize()
+            ts = []
+            for _ in range(reps):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                mp.mp_master_update(plan, st, opt, mode)
+                b.record()
+                mp.mp_loss_scale_update(st)
+                ts.append((a, b))
+            torch.cuda.synchronize()
+            return sum(a.elapsed_time(b) for a, b in ts) / reps
+        ms0 = timed(0, iters)
+        ms1 = timed(1, iters)
+        g16.view(torch.int16)[offs[-1] + counts[-1] - 1] = 0x7C00      # overflow: skipped steps
+        ms_skip = timed(1, iters)
+        assert st.read().skipped >= iters
+        rows.append({"params": P, "tensors": n, "ms_trusted_flag": ms0, "gbs_28B": P * 28 / ms0 / 1e6,
+                     "ms_with_inspection": ms1, "gbs_28B_with_inspection": P * 28 / ms1 / 1e6,
+                     "gbs_30B_moved_with_inspection": P * 30 / ms1 / 1e6, "ms_skipped_step": ms_skip,
+                     "note": "L2-resident / launch-bound" if P * 16 < 126e6 else "HBM-bound"})
+        plan.close()
+        st.close()
+        del g16, w16, w32, m, v, z
+        torch.cuda.empty_cache()
+    clocks = sampler.stop()
+    top = rows[-1]
+    print(json.dumps({
+        "metric": METRIC, "value": top["gbs_28B"], "unit": "GB/s", "n_gpus": 1, "steps": args.steps,
+        "warmup": 3, "ms_per_step": top["ms_trusted_flag"], "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f16 gradients / f32 master", "data": "synthetic",
+        "config": {"workload": "c5: update-only sweep, Adam, 1e6..1e9 parameters in 1..500 log-uniform tensors",
+                   "cache": "1e8 and 1e9 parameters (1.6 / 16 GB of state) far exceed the 126 MB L2"},
+        "gpu_launches": int(mp.mp_kernel_launch_count() - launches0),
+        "roofline": {"kernel": "mp_master_update_kernel", "bound": "hbm", "achieved": top["gbs_28B"],
+                     "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": top["gbs_28B"] / pk["hbm_gbs"],
+                     "traffic": None, "peak_source": pk_src + " copy", "frac_of_nominal_8000": top["gbs_28B"] / 8000.0},
+        "sweep": rows, "clocks": clocks}))
+
+
 # ------------------------------------------------------------------ CUDA arm
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=10)
-    ap.add_argument("--workload", default="c2", choices=["c2", "c3", "c4"])
+    ap.add_argument("--workload", default="c2", choices=["c2", "c3", "c4", "c5"])
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
+    if args.workload == "c5":
+        return run_update_sweep(args)
 
     import numpy as np
     import torch

@@ -85,11 +85,15 @@ class StackConfig:
     steps: int = 3
     inject_inf_step: int = -1        # 0-based step whose top gradient gets a +inf
     note: str = ""
+    chain: list = field(default_factory=list)   # per layer: reads the previous layer's output
 
     def chained(self, l: int) -> bool:
-        """Layer l reads layer l-1's output when the widths line up."""
-        return l > 0 and self.shapes[l][1] == self.shapes[l - 1][2] and \
+        """Layer l reads layer l-1's output (needs matching widths and rows).  Without an
+        explicit `chain` list every layer whose input width equals the previous output width
+        is chained."""
+        fits = l > 0 and self.shapes[l][1] == self.shapes[l - 1][2] and \
             self.shapes[l][0] == self.shapes[l - 1][0]
+        return fits and (self.chain[l] if self.chain else True)
 
     def feeds_next(self, l: int) -> bool:
         return l + 1 < len(self.shapes) and self.chained(l + 1)
@@ -113,24 +117,15 @@ def config(name: str) -> StackConfig:
                            note="8 layers, 128x50 tokens, 2048->4096; lr from the paper's listing")
     if name == "c3":      # Transformer-big FFN pair + 4 attention projections per block
         blk = [(8192, 1024, 4096), (8192, 4096, 1024)] + [(8192, 1024, 1024)] * 4
+        # only the FFN pair is chained; the four attention projections are independent layers
         return StackConfig("c3", 2, blk * 6, grad_std=10 ** -2.5, init_scale=2.0 ** 15,
+                           chain=[False, True, False, False, False, False] * 6,
                            note="6 blocks x (FFN 1024->4096->1024 + 4 proj 1024x1024), 8192 tokens")
     if name == "c4":      # DeepSpeech2-like dense stack, momentum SGD, heavy-tailed inputs
         return StackConfig("c4", 3, [(25600, 1600, 1600)] * 5 + [(25600, 1600, 29)],
-                           optimizer="momentum", grad_std=1e-3, x_dist="lognormal2",
+                           optimizer="momentum", lr=1e-7, grad_std=1e-3, x_dist="lognormal2",
                            note="5 x 1600->1600 over 64x400 frames + 1600->29")
     raise KeyError(name)
-
-
-def small_variant(cfg: StackConfig, rows: int, div: int) -> StackConfig:
-    """Same recipe with rows and widths shrunk (kept multiples of 8), for oracle-sized parity."""
-    def r8(v):
-        return max(8, (v // div + 7) // 8 * 8) if v > 64 else v
-    shapes = [(rows, r8(k), r8(n)) for _, k, n in cfg.shapes]
-    out = StackConfig(**{**cfg.__dict__})
-    out.shapes = shapes
-    out.name = cfg.name + "_small"
-    return out
 
 
 def weights(cfg: StackConfig, l: int) -> np.ndarray:
