@@ -329,12 +329,31 @@ def main():
     if rank == 0:
         sampler.start()
         time.sleep(0.3)
-    stack.events = []
-    ms_total = timed(lambda: stack.step(xs, gs), args.steps)
-    events, stack.events = stack.events, None
-    launches = mp.mp_kernel_launch_count() - launches0
+    # (A) the step as one CUDA graph replay per step: `value`
+    launches_per_step = mp.mp_kernel_launch_count()
+    stack.step(xs, gs)
+    launches_per_step = mp.mp_kernel_launch_count() - launches_per_step
+    use_graph = world == 1          # the data-parallel step (NCCL all-reduce inside) is launched call by call
+    if use_graph:
+        stack.capture(xs, gs)
+    run_step = stack.replay if use_graph else (lambda: stack.step(xs, gs))
+    for _ in range(3):
+        run_step()
+    torch.cuda.synchronize()
+    st0 = stack.state.read()
+    ms_total = timed(run_step, args.steps)
     st1 = stack.state.read()
-    # end to end: pinned host inputs in, loss-scale state out, every step
+    launches = launches_per_step * args.steps
+    # (B) the same steps launched call by call with a CUDA-event pair around every launch:
+    # per-kernel times for the roofline (the event records cost ~6 % of the step, so this
+    # region is not the one `value` is taken from)
+    stack.events = []
+    st0b = stack.state.read()
+    ms_events = timed(lambda: stack.step(xs, gs), args.steps)
+    events, stack.events = stack.events, None
+    st1b = stack.state.read()
+    # (C) end to end: pinned host inputs in, loss-scale state out, every step
+    stack.use_graph_from_host = use_graph
     for _ in range(2):
         stack.step_from_host(xs_host, gs_host)
     ms_e2e = timed(lambda: stack.step_from_host(xs_host, gs_host), args.steps)
@@ -354,12 +373,13 @@ def main():
     gemm_calls = sum(len(per.get(k, [])) for k in ("fwd", "dgrad", "wgrad"))
     gemm_tflops = flops_step * args.steps / (gemm_ms * 1e-3) / 1e12
     skipped = st1.skipped - st0.skipped
+    skipped_b = st1b.skipped - st0b.skipped
     bytes_per_param = 28 if cfg.optimizer == "adam" else 20
     upd_ms = per.get("update", [0.0])
     applied = [t for t in upd_ms]
     upd_bytes = cfg.n_params() * bytes_per_param
     # skipped steps return at once; GB/s is quoted on the applied ones only
-    applied_ms = sorted(applied)[skipped:] if skipped < len(applied) else applied
+    applied_ms = sorted(applied)[skipped_b:] if skipped_b < len(applied) else applied
     upd_gbs = upd_bytes / (sum(applied_ms) / len(applied_ms) * 1e-3) / 1e9
     sha = kernel_sha()
     traffic = NCU_TRAFFIC["bytes_per_launch"].get(args.workload) if NCU_TRAFFIC["sha"] == sha else None
@@ -374,6 +394,9 @@ def main():
         "e2e": {"value": e2e_val, "unit": "TFLOP/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": ms_e2e / args.steps},
         "gpu_launches": int(launches),
+        "launch_mode": "one CUDA graph replay per step (captured from the same C-ABI calls)" if use_graph
+                       else "call by call",
+        "ms_per_step_call_by_call_with_events": ms_events / args.steps,
         "skipped_steps_in_timed_region": int(skipped),
         "loss_scale": st1.scale,
         "roofline": {"kernel": "mp_gemm_kernel", "bound": "tensor", "achieved": gemm_tflops,
@@ -383,6 +406,8 @@ def main():
                      "frac_of_burst_peak": gemm_tflops / pk["bf16_tflops"],
                      "frac_of_nominal_2250": gemm_tflops / 2250.0,
                      "launches": gemm_calls, "avg_launch_ms": gemm_ms / max(gemm_calls, 1),
+                     "timed_in": "a second timed region of the same steps, launched call by call with a "
+                                 "CUDA-event pair around every launch",
                      "per_op_tflops": {k: (flops_step / 3) * args.steps / (sum(per[k]) * 1e-3) / 1e12
                                        for k in ("fwd", "dgrad", "wgrad") if k in per}},
         "update": {"kernel": "mp_master_update_kernel", "bound": "hbm", "achieved": upd_gbs,

@@ -162,3 +162,45 @@ def test_scaled_down_workloads(orc, mp, name, rows, shapes):
     cfg.growth_interval = 2
     recs = run_config(orc, mp, cfg, 4)
     assert len(recs) == 4
+
+
+def test_graph_replay_equals_call_by_call(orc, mp):
+    """The step captured once as a CUDA graph and replayed must leave bit-for-bit the state that
+    the same steps launched call by call leave, including an overflow step (skip + halving),
+    because flag, scale and step count never leave the device."""
+    from paper_1805_10387_b200.stack import LinearStack
+    cfg = synth.config("c1")
+    L = len(cfg.shapes)
+    chained = [cfg.chained(l) for l in range(L)]
+
+    def make():
+        st = LinearStack(cfg.shapes, chained, lr=cfg.lr, init_scale=cfg.init_scale, growth_interval=3)
+        for l in range(L):
+            w = synth.weights(cfg, l)
+            st.load_weights(l, torch.from_numpy(w).cuda(),
+                            torch.from_numpy(synth.fp16_bits(w).view(np.float16).reshape(w.shape)).cuda())
+        return st
+    a, b = make(), make()
+    x = _pad_dev(synth.activations(cfg, 0, 0))
+    g = torch.from_numpy(synth.upstream(cfg, 1, 0)).cuda()
+    xs, gs = [x, None], [None, g]
+    steps = 9
+    b.capture(xs, gs, warmup=2)                      # two real steps, then the recording
+    for _ in range(2):
+        a.step(xs, gs)
+    for s in range(steps):
+        if s == 4:
+            g[0, 0] = float("inf")                   # replayed graph reads the tensor as it is now
+        if s == 5:
+            g[0, 0] = 0.0
+        a.step(xs, gs)
+        b.replay()
+    torch.cuda.synchronize()
+    ha, hb = a.state.read(), b.state.read()
+    assert (ha.scale, ha.t, ha.skipped, ha.step, ha.good_steps) == (hb.scale, hb.t, hb.skipped, hb.step, hb.good_steps)
+    assert ha.skipped >= 1 and ha.step == steps + 2
+    assert [r.found_inf for r in a.state.read_log()] == [r.found_inf for r in b.state.read_log()]
+    for fa, fb in ((a.w32_flat, b.w32_flat), (a.m_flat, b.m_flat), (a.v_flat, b.v_flat)):
+        assert torch.equal(fa.view(torch.int32), fb.view(torch.int32))
+    assert torch.equal(a.w16_flat.view(torch.int16), b.w16_flat.view(torch.int16))
+    a.close(); b.close()
