@@ -32,7 +32,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 
 # DRAM bytes per launch of the GEMM kernel from one ncu capture (dram__bytes_read.sum +
 # dram__bytes_write.sum), keyed by workload, valid only for the kernel source it was taken on.
-NCU_TRAFFIC = {"sha": "848deb081eb53860", "bytes_per_launch": {"c2": 50.7e6}}
+NCU_TRAFFIC = {"sha": "1e34a6610b121c20", "bytes_per_launch": {"c2": 53.0e6}}
 
 
 def peaks():
