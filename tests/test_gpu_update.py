@@ -285,3 +285,81 @@ def test_sweep_workload_trajectory(orc, mp):
     assert (np.abs(w - w_host)[live] <= 1e-6 * np.maximum(np.abs(w_host[live]), 1e-3)).all()
     assert (_bits(T.w16)[live] == w16_host[live]).mean() > 0.9999
     st.close(); plan.close()
+
+
+@pytest.mark.parametrize("kind", ["adam", "momentum"])
+def test_weight_decay_on_the_master_copy(orc, mp, kind):
+    """Section 3.3: the decay term is formed from the FP32 master and added to the FP32 gradient.
+    With a coefficient of 1e-5 and weights near 5e-4 the product is below FP16's smallest
+    subnormal, so a decay formed in FP16 would vanish; here it must move the weights."""
+    n = 12345
+    adam = kind == "adam"
+    rng = np.random.default_rng(8)
+    T = Tensors([n], adam)
+    w0 = (rng.standard_normal(n) * 5e-4).astype(np.float32)
+    T.w32[:n] = torch.from_numpy(w0).cuda()
+    host = dict(w32=w0.copy(), m=np.zeros(n, np.float32), v=np.zeros(n, np.float32), w16=np.zeros(n, np.uint16))
+    plan = T.plan(mp)
+    st = mp.State(init_scale=256.0, growth_interval=1000)
+    wd = 1e-5
+    assert ((orc.f2h((wd * w0).astype(np.float32)) & 0x7FFF) == 0).mean() > 0.99   # lost in FP16
+    opt = mp.OptimConfig(mp.MP_OPT_ADAM if adam else mp.MP_OPT_MOMENTUM, 1e-2, 0.9, 0.999, 1e-8, 0.9, wd)
+    zero_g = np.zeros(n, np.uint16)                                        # gradient exactly zero
+    for step in range(4):
+        T.g16[:n] = _dev16(zero_g)
+        mp.mp_master_update(plan, st, opt, 1)
+        mp.mp_loss_scale_update(st)
+        if adam:
+            orc.adam_update(zero_g, host["w32"], host["m"], host["v"], host["w16"], 256.0, 1e-2, 0.9, 0.999,
+                            1e-8, step + 1, wd)
+        else:
+            orc.momentum_update(zero_g, host["w32"], host["m"], host["w16"], 256.0, 1e-2, 0.9, wd)
+    w = T.w32[:n].cpu().numpy()
+    assert (np.abs(w - host["w32"]) <= 1e-6 * np.maximum(np.abs(host["w32"]), 1e-3)).all()
+    moved = np.abs(w - w0) > 0
+    assert moved.mean() > 0.99                                             # the decay acted
+    if not adam:                                                           # plain decay shrinks weights
+        assert (np.sign(w0 - w)[moved] == np.sign(w0)[moved]).all() and (np.abs(w) < np.abs(w0))[moved].all()
+    assert (_bits(T.w16[:n]) == orc.f2h(w)).all()
+    st.close(); plan.close()
+
+
+def test_state_checkpoint_and_resume(orc, mp):
+    """Ten steps in one go equal five steps, a state export / import into fresh objects, and five
+    more steps, bit for bit (loss scale, counters, master weights, moments)."""
+    rng = np.random.default_rng(9)
+    n = 50000
+    w0 = rng.standard_normal(n).astype(np.float32)
+    grads = [(rng.standard_normal(n) * 300.0).astype(np.float16) for _ in range(10)]
+    grads[3][17] = np.inf
+    opt = mp.OptimConfig(mp.MP_OPT_ADAM, 1e-3, 0.9, 0.999, 1e-8, 0.9, 0.0)
+
+    def fresh():
+        T = Tensors([n])
+        T.w32[:n] = torch.from_numpy(w0).cuda()
+        return T, T.plan(mp), mp.State(init_scale=1024.0, growth_interval=2)
+
+    def run(T, plan, st, lo, hi):
+        for s in range(lo, hi):
+            T.g16[:n] = torch.from_numpy(grads[s]).cuda()
+            mp.mp_master_update(plan, st, opt, 1)
+            mp.mp_loss_scale_update(st)
+    Ta, pa, sa = fresh()
+    run(Ta, pa, sa, 0, 10)
+    Tb, pb, sb = fresh()
+    run(Tb, pb, sb, 0, 5)
+    snap = sb.read()                                           # export
+    saved = [x.clone() for x in (Tb.w32, Tb.m, Tb.v, Tb.w16)]
+    Tc, pc, sc2 = fresh()                                      # import into new objects
+    for dst, src in zip((Tc.w32, Tc.m, Tc.v, Tc.w16), saved):
+        dst.copy_(src)
+    sc2.write(snap)
+    run(Tc, pc, sc2, 5, 10)
+    ha, hc = sa.read(), sc2.read()
+    assert (ha.scale, ha.t, ha.step, ha.skipped, ha.good_steps) == (hc.scale, hc.t, hc.step, hc.skipped, hc.good_steps)
+    assert ha.skipped == 1
+    for x, y in zip((Ta.w32, Ta.m, Ta.v), (Tc.w32, Tc.m, Tc.v)):
+        assert torch.equal(x.view(torch.int32), y.view(torch.int32))
+    assert torch.equal(Ta.w16.view(torch.int16), Tc.w16.view(torch.int16))
+    for s_, p_ in ((sa, pa), (sb, pb), (sc2, pc)):
+        s_.close(); p_.close()
