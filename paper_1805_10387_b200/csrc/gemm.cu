@@ -144,6 +144,7 @@ mp_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                                              ~static_cast<uintptr_t>(1023));
   Barriers* bars = reinterpret_cast<Barriers*>(smem + STAGES * STAGE_BYTES);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  ptx::launch_dependents();    // the next kernel's CTAs may take SMs as soon as ours leave them
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
@@ -167,6 +168,9 @@ mp_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   __syncthreads();
   ptx::tc_fence_after_sync();
   const uint32_t tmem_base = bars->tmem_base;
+  // Everything above (barriers, tensor memory, descriptor prefetch) may overlap the tail of the
+  // previous kernel in the stream; nothing below may.
+  ptx::grid_dependency_wait();
 
   const int total_work = p.m_tiles * p.n_tiles * p.splits;
 
@@ -325,6 +329,7 @@ mp_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a,
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = ptx::cluster_ctarank();
   const bool leader = rank == 0;
+  ptx::launch_dependents();    // the next kernel's CTAs may take SMs as soon as ours leave them
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES2; ++s) {
@@ -349,6 +354,8 @@ mp_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a,
   ptx::cluster_sync();                              // both CTAs' barriers exist before any remote arrive
   ptx::tc_fence_after_sync();
   const uint32_t tmem_base = bars->tmem_base;
+  // Everything above may overlap the tail of the previous kernel in the stream; nothing below may.
+  ptx::grid_dependency_wait();
 
   const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
   const int total_work = p.m_tiles * p.n_tiles * p.splits;   // m_tiles counts 256-row tiles here
@@ -596,9 +603,18 @@ int launch(const CUtensorMap& ma, const CUtensorMap& mb, const GemmParams& p, in
                                      cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
     attr_set = true;
   }
-  mp_gemm_kernel<A_MN, B_MN><<<grid, THREADS, SMEM_BYTES, st>>>(ma, mb, p);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid, 1, 1);
+  cfg.blockDim = dim3(THREADS, 1, 1);
+  cfg.dynamicSmemBytes = SMEM_BYTES;
+  cfg.stream = st;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  MP_CUDA_TRY(cudaLaunchKernelEx(&cfg, mp_gemm_kernel<A_MN, B_MN>, ma, mb, p));
   mp::count_launch();
-  MP_CUDA_TRY(cudaGetLastError());
   return MP_OK;
 }
 
@@ -624,9 +640,18 @@ int launch_pair(const CUtensorMap& ma, const CUtensorMap& mb, const GemmParams& 
     max_pairs = n;
   }
   const int pairs = (int)(work < max_pairs ? work : max_pairs);
-  mp_gemm_pair_kernel<A_MN, B_MN><<<2 * pairs, THREADS, SMEM2_BYTES, st>>>(ma, mb, p);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2 * pairs, 1, 1);
+  cfg.blockDim = dim3(THREADS, 1, 1);
+  cfg.dynamicSmemBytes = SMEM2_BYTES;
+  cfg.stream = st;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  MP_CUDA_TRY(cudaLaunchKernelEx(&cfg, mp_gemm_pair_kernel<A_MN, B_MN>, ma, mb, p));
   mp::count_launch();
-  MP_CUDA_TRY(cudaGetLastError());
   return MP_OK;
 }
 

@@ -211,6 +211,19 @@ __device__ __forceinline__ void mma_commit_pair(uint64_t* bar, uint16_t cta_mask
       : "memory");
 }
 
+// ---- programmatic dependent launch ----------------------------------------------------------
+// A kernel launched with the programmatic-stream-serialization attribute may start while the
+// kernel before it in the stream is still running, once every CTA of that kernel has executed
+// launch_dependents (or exited).  It must execute grid_dependency_wait before it touches
+// memory the earlier kernel reads or writes: that returns when the earlier kernel has
+// completed and its writes are visible.
+__device__ __forceinline__ void launch_dependents() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+__device__ __forceinline__ void grid_dependency_wait() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 // ---- descriptors ----------------------------------------------------------------------
 // Shared-memory matrix descriptor, 128-byte swizzle.  Bits: [0,14) start address >> 4,
 // [16,30) leading byte offset >> 4, [32,46) stride byte offset >> 4, [46,48) = 1 (sm_100
