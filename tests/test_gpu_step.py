@@ -23,13 +23,13 @@ def _pad_dev(bits):
     return buf
 
 
-def build_both(orc, cfg):
+def build_both(orc, cfg, dynamic=True):
     from paper_1805_10387_b200.stack import LinearStack
     L = len(cfg.shapes)
     chained = [cfg.chained(l) for l in range(L)]
     gpu = LinearStack(cfg.shapes, chained, optimizer=cfg.optimizer, lr=cfg.lr, beta1=cfg.beta1,
                       beta2=cfg.beta2, eps=cfg.eps, momentum=cfg.momentum,
-                      init_scale=cfg.init_scale, growth_interval=cfg.growth_interval)
+                      init_scale=cfg.init_scale, growth_interval=cfg.growth_interval, dynamic=dynamic)
     layers = []
     for l in range(L):
         w = synth.weights(cfg, l)
@@ -38,7 +38,7 @@ def build_both(orc, cfg):
         gpu.load_weights(l, torch.from_numpy(w).cuda(),
                          torch.from_numpy(synth.fp16_bits(w).view(np.float16).reshape(w.shape)).cuda())
         assert (synth.fp16_bits(w).reshape(w.shape) == ly.w16).all()
-    sc = orc.Scaler(cfg.init_scale, cfg.growth_interval)
+    sc = orc.Scaler(cfg.init_scale, cfg.growth_interval, dynamic=dynamic)
     opt = orc.Optim(kind=cfg.optimizer, lr=cfg.lr, beta1=cfg.beta1, beta2=cfg.beta2, eps=cfg.eps,
                     momentum=cfg.momentum)
     return gpu, layers, sc, opt
@@ -78,8 +78,8 @@ def forced_ok(orc, op, A_bits, B_bits, got_bits, what):
             assert (np.abs(g[big] - w[big]) / np.abs(w[big])).max() <= 1e-2, what
 
 
-def run_config(orc, mp, cfg, steps):
-    gpu, layers, sc, opt = build_both(orc, cfg)
+def run_config(orc, mp, cfg, steps, dynamic=True):
+    gpu, layers, sc, opt = build_both(orc, cfg, dynamic)
     L = len(cfg.shapes)
     records = []
     for step in range(steps):
@@ -146,6 +146,17 @@ def test_c1_ten_steps_with_injected_inf(orc, mp):
     recs = run_config(orc, mp, cfg, cfg.steps)
     assert [r.found_inf for r in recs] == [0, 0, 0, 0, 1, 0, 0, 0, 0, 0]
     assert [np.log2(r.S_after) for r in recs] == [16, 16, 16, 17, 16, 16, 16, 16, 17, 17]
+
+
+def test_static_loss_scale_that_is_not_a_power_of_two(orc, mp):
+    """Static loss scaling with the value of the paper's configuration listing (10.0): S never
+    changes, the unscale is a multiply by fl32(1/10), the step with the injected inf is still
+    skipped, and everything matches the oracle as in the dynamic case."""
+    cfg = synth.config("c1")
+    cfg.init_scale = 10.0
+    recs = run_config(orc, mp, cfg, 7, dynamic=False)
+    assert [r.found_inf for r in recs] == [0, 0, 0, 0, 1, 0, 0]
+    assert all(r.S_before == 10.0 and r.S_after == 10.0 for r in recs)
 
 
 @pytest.mark.parametrize("name,rows,shapes", [
