@@ -208,6 +208,64 @@ void orc_linear_exact(int op, const uint16_t* A, int64_t lda, const uint16_t* B,
   });
 }
 
+// ------------------------------------------- layers with bias and activation
+// The paper's models put a bias and a nonlinearity after their dense products (ReLU in the
+// Transformer feed-forward block, clipped ReLU in DeepSpeech2; Section 5).  Readings, since the
+// paper states none: the bias is added to the FP32 sum before the one rounding to FP16; the
+// activation acts on that FP32 value; the backward pass masks the FP16 data gradient with the
+// derivative taken from the stored FP16 output (1 where the output is strictly inside the
+// activation's linear range, else 0).
+// act: 0 identity, 1 max(x,0), 2 min(max(x,0),clip).
+static inline float apply_act(float x, int act, float clip) {
+  if (act == 1) return x > 0.0f ? x : 0.0f;
+  if (act == 2) { x = x > 0.0f ? x : 0.0f; return x < clip ? x : clip; }
+  return x;
+}
+static inline bool act_passes(float y, int act, float clip) {
+  if (act == 1) return y > 0.0f;
+  if (act == 2) return y > 0.0f && y < clip;
+  return true;
+}
+
+// Y[m,n] = rn16( act( sum_k X[m,k] W[k,n] + b[n] ) ); b may be null.
+void orc_linear_fwd_act(const uint16_t* X, int64_t ldx, const uint16_t* W, int64_t ldw,
+                        const uint16_t* b, uint16_t* Y, int64_t ldy, int64_t M, int64_t K,
+                        int64_t N, int act, float clip, int nthreads) {
+  parallel_rows(M, nthreads, [=](int64_t lo, int64_t hi) {
+    for (int64_t m = lo; m < hi; ++m)
+      for (int64_t n = 0; n < N; ++n) {
+        float acc = 0.0f;
+        for (int64_t k = 0; k < K; ++k) acc = acc + h2f(X[m * ldx + k]) * h2f(W[k * ldw + n]);
+        if (b) acc = acc + h2f(b[n]);
+        Y[m * ldy + n] = f2h(apply_act(acc, act, clip));
+      }
+  });
+}
+
+// dX[m,k] = rn16( sum_n dY[m,n] W[k,n] ) where the layer's input A[m,k] (the previous layer's
+// activated output) lies strictly inside the linear range of that layer's activation, else +0.
+void orc_linear_bwd_dgrad_act(const uint16_t* dY, int64_t lddy, const uint16_t* W, int64_t ldw,
+                              const uint16_t* A, int64_t lda, uint16_t* dX, int64_t lddx,
+                              int64_t M, int64_t K, int64_t N, int act, float clip, int nthreads) {
+  parallel_rows(M, nthreads, [=](int64_t lo, int64_t hi) {
+    for (int64_t m = lo; m < hi; ++m)
+      for (int64_t k = 0; k < K; ++k) {
+        float acc = 0.0f;
+        for (int64_t n = 0; n < N; ++n) acc = acc + h2f(dY[m * lddy + n]) * h2f(W[k * ldw + n]);
+        dX[m * lddx + k] = act_passes(h2f(A[m * lda + k]), act, clip) ? f2h(acc) : (uint16_t)0;
+      }
+  });
+}
+
+// db[n] = rn16( sum_m dY[m,n] ), FP32 running sum, m ascending (still multiplied by S).
+void orc_bias_grad(const uint16_t* dY, int64_t lddy, uint16_t* db, int64_t M, int64_t N) {
+  for (int64_t n = 0; n < N; ++n) {
+    float acc = 0.0f;
+    for (int64_t m = 0; m < M; ++m) acc = acc + h2f(dY[m * lddy + n]);
+    db[n] = f2h(acc);
+  }
+}
+
 // ----------------------------------------------------- upstream scaling (O3)
 // Section 3.1 item 1: the loss (here: the gradient entering the top layer) is
 // multiplied by the current scale S, in FP32, then stored as FP16.

@@ -57,6 +57,9 @@ def lib():
             getattr(L, name).restype = None
         L.orc_linear_sampled.argtypes = [i32, p, i64, p, i64, i64, i64, i64, p, p, i64, p, p, p]
         L.orc_linear_exact.argtypes = [i32, p, i64, p, i64, i64, i64, i64, p, p, i32]
+        L.orc_linear_fwd_act.argtypes = [p, i64, p, i64, p, p, i64, i64, i64, i64, i32, f32, i32]
+        L.orc_linear_bwd_dgrad_act.argtypes = [p, i64, p, i64, p, i64, p, i64, i64, i64, i64, i32, f32, i32]
+        L.orc_bias_grad.argtypes = [p, i64, p, i64, i64]
         L.orc_scale_upstream.argtypes = [p, f32, p, i64]
         L.orc_found_inf.restype = i32; L.orc_found_inf.argtypes = [p, i64]
         L.orc_adam_update.argtypes = [p, p, p, p, p, i64, f32, f32, f32, f32, f32, f32, i64]
@@ -124,6 +127,40 @@ def linear_bwd_wgrad(X16, dY16, nthreads=0) -> np.ndarray:
     lib().orc_linear_bwd_wgrad(_ptr(X16), K, _ptr(dY16), N, _ptr(dW), N, M, K, N,
                                nthreads or hardware_threads())
     return dW
+
+
+ACT = {"none": 0, "relu": 1, "clipped_relu": 2}
+
+
+def linear_fwd_act(X16, W16, b16=None, act="none", clip=20.0, nthreads=0) -> np.ndarray:
+    """Y = rn16(act(X W + b)): bias added to the FP32 sum, activation on the FP32 value."""
+    _chk(X16, np.uint16); _chk(W16, np.uint16)
+    M, K = X16.shape; K2, N = W16.shape; assert K == K2
+    if b16 is not None:
+        _chk(b16, np.uint16); assert b16.shape == (N,)
+    Y = np.empty((M, N), np.uint16)
+    lib().orc_linear_fwd_act(_ptr(X16), K, _ptr(W16), N, _ptr(b16) if b16 is not None else None,
+                             _ptr(Y), N, M, K, N, ACT[act], clip, nthreads or hardware_threads())
+    return Y
+
+
+def linear_bwd_dgrad_act(dY16, W16, A16, act="none", clip=20.0, nthreads=0) -> np.ndarray:
+    """dX = rn16(dY W^T) masked by the derivative of `act` at the layer input A (FP16 [M,K])."""
+    _chk(dY16, np.uint16); _chk(W16, np.uint16); _chk(A16, np.uint16)
+    M, N = dY16.shape; K, N2 = W16.shape; assert N == N2 and A16.shape == (M, K)
+    dX = np.empty((M, K), np.uint16)
+    lib().orc_linear_bwd_dgrad_act(_ptr(dY16), N, _ptr(W16), N, _ptr(A16), K, _ptr(dX), K, M, K, N,
+                                   ACT[act], clip, nthreads or hardware_threads())
+    return dX
+
+
+def bias_grad(dY16) -> np.ndarray:
+    """db[n] = rn16(sum_m dY[m,n]), FP32 running sum."""
+    _chk(dY16, np.uint16)
+    M, N = dY16.shape
+    db = np.empty(N, np.uint16)
+    lib().orc_bias_grad(_ptr(dY16), N, _ptr(db), M, N)
+    return db
 
 
 _OPS = {"fwd": 0, "dgrad": 1, "wgrad": 2}
