@@ -161,6 +161,38 @@ int mp_linear_bwd_wgrad_static(const void* X16, int64_t ldx, const void* dY16, i
 /* Size of that built-in scratch in bytes (equals MP_STATIC_SCRATCH_BYTES). */
 size_t mp_static_scratch_bytes(void);
 
+/* ---- layers with a bias and an activation ------------------------------------------------
+ * The models of the paper's Section 5 follow their dense products with a bias and a
+ * nonlinearity (ReLU in the Transformer feed-forward block, clipped ReLU in DeepSpeech2).  The
+ * paper gives no arithmetic for them; this library's reading: the FP16 bias is added to the
+ * FP32 sum before the single rounding to FP16, the activation acts on that FP32 value, and the
+ * backward pass zeroes the FP16 data gradient where the stored FP16 output of the activated
+ * layer is outside the activation's linear range. */
+typedef enum { MP_ACT_NONE = 0, MP_ACT_RELU = 1, MP_ACT_CLIPPED_RELU = 2 } mp_activation;
+
+/* Y[M,N] = rn16( act( sum_k X[m,k] W[k,n] + bias[n] ) ).  bias16: N FP16 values, 16-byte aligned,
+ * or NULL.  act: mp_activation; clip: upper bound of MP_ACT_CLIPPED_RELU (min(max(x,0),clip)).
+ * Other arguments and errors as mp_linear_fwd. */
+int mp_linear_fwd_act(const void* X16, int64_t ldx, const void* W16, int64_t ldw, const void* bias16,
+                      void* Y16, int64_t ldy, int64_t M, int64_t K, int64_t N, int act, float clip,
+                      void* workspace, size_t workspace_bytes, void* stream);
+
+/* dX[m,k] = rn16( sum_n dY[m,n] W[k,n] ) where A[m,k] passes the activation (A > 0 for ReLU,
+ * 0 < A < clip for clipped ReLU), else +0.  A16 [M,K] (lda >= K) is this layer's input, i.e.
+ * the activated FP16 output of the layer below; it may alias nothing that is written.  With
+ * MP_ACT_NONE the call equals mp_linear_bwd_dgrad and A16 may be NULL. */
+int mp_linear_bwd_dgrad_act(const void* dY16, int64_t lddy, const void* W16, int64_t ldw,
+                            const void* A16, int64_t lda, void* dX16, int64_t lddx, int64_t M,
+                            int64_t K, int64_t N, int act, float clip, void* workspace,
+                            size_t workspace_bytes, void* stream);
+
+/* db[n] = rn16( sum_m dY[m,n] ), FP32 accumulation in a fixed order (results do not depend on
+ * timing), still multiplied by S.  Sets state->found_inf if a stored value is inf or NaN (state
+ * may be NULL).  workspace: at least mp_bias_grad_workspace_bytes(M,N) bytes of device scratch. */
+int mp_bias_grad(const void* dY16, int64_t lddy, void* db16, int64_t M, int64_t N, mp_state* state,
+                 void* workspace, size_t workspace_bytes, void* stream);
+size_t mp_bias_grad_workspace_bytes(int64_t M, int64_t N);
+
 /* ---- auxiliaries --------------------------------------------------------------------- */
 
 enum { MP_OP_FWD = 0, MP_OP_DGRAD = 1, MP_OP_WGRAD = 2 };

@@ -52,6 +52,15 @@ struct GemmParams {
   float* ws;            // FP32 partials [splits][Mo][ws_ld]
   int64_t ws_ld;
   int* flag;            // found_inf word, or null
+  // Optional fused epilogue (FP16 output only).  Forward flavour: add bias[col] to the FP32 sum,
+  // then the activation.  Data-gradient flavour: zero the output where the layer input
+  // mask[row, col] (the previous layer's activated FP16 output) is outside the activation's
+  // linear range.  act: 0 none, 1 max(x,0), 2 min(max(x,0),clip).
+  const uint16_t* bias;
+  const uint16_t* mask;
+  int64_t ldmask;
+  int act;
+  float clip;
 };
 
 struct Barriers {
@@ -103,11 +112,38 @@ __device__ __forceinline__ uint32_t epilogue_tile(const GemmParams& p, uint32_t 
         }
       }
     } else {
+      if (p.bias != nullptr || (p.act != 0 && p.mask == nullptr)) {
+        // forward flavour, on the FP32 values: + bias, then the activation
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          float x = __uint_as_float(r[j]);
+          if (p.bias != nullptr && col0 + j < p.No)
+            x = __fadd_rn(x, __half2float(__ushort_as_half(__ldg(p.bias + col0 + j))));
+          if (p.act != 0) {
+            x = x > 0.0f ? x : 0.0f;
+            if (p.act == 2) x = x < p.clip ? x : p.clip;
+          }
+          r[j] = __float_as_uint(x);
+        }
+      }
       uint32_t h[16];
 #pragma unroll
       for (int j = 0; j < 16; ++j) {
         const __half2 v = __floats2half2_rn(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1]));
         h[j] = *reinterpret_cast<const uint32_t*>(&v);
+      }
+      if (p.mask != nullptr && p.act != 0 && row_ok) {
+        // data-gradient flavour: keep the value only where the layer input passes the activation
+        const uint16_t* mrow = p.mask + (int64_t)row * p.ldmask + col0;
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          bool pass = false;
+          if (col0 + j < p.No) {
+            const float y = __half2float(__ushort_as_half(__ldg(mrow + j)));
+            pass = p.act == 2 ? (y > 0.0f && y < p.clip) : (y > 0.0f);
+          }
+          if (!pass) h[j >> 1] &= (j & 1) ? 0x0000FFFFu : 0xFFFF0000u;
+        }
       }
       if (row_ok) {
         uint16_t* dst = p.out + (int64_t)row * p.ldo + col0;
@@ -587,6 +623,14 @@ int choose_splits(int64_t Mo, int64_t No, int64_t R) {
 
 int64_t ws_ld_for(int64_t No) { return (No + 3) / 4 * 4; }
 
+struct Fuse {
+  const void* bias = nullptr;
+  const void* mask = nullptr;
+  int64_t ldmask = 0;
+  int act = 0;
+  float clip = 0.0f;
+};
+
 struct Operand {
   const void* ptr;
   int64_t ld;
@@ -656,7 +700,8 @@ int launch_pair(const CUtensorMap& ma, const CUtensorMap& mb, const GemmParams& 
 }
 
 int run_gemm(const char* name, const Operand& A, const Operand& B, void* out, int64_t ldo,
-             int* flag, bool want_flag, void* workspace, size_t ws_bytes, cudaStream_t st) {
+             int* flag, bool want_flag, void* workspace, size_t ws_bytes, cudaStream_t st,
+             const Fuse& fuse = Fuse()) {
   const int64_t Mo = A.mn, No = B.mn, R = A.red;
   if (!A.ptr || !B.ptr || !out) return mp::set_error(MP_ERR_INVALID_ARG, "%s: null pointer", name);
   if (Mo <= 0 || No <= 0 || R <= 0)
@@ -680,7 +725,10 @@ int run_gemm(const char* name, const Operand& A, const Operand& B, void* out, in
   p.m_tiles = (int)(pair ? (Mo + 255) / 256 : (Mo + BM - 1) / BM);
   p.n_tiles = (int)((No + BN - 1) / BN);
   p.num_kb = (int)((R + BK - 1) / BK);
-  p.splits = choose_splits(Mo, No, R);
+  const bool fused = fuse.bias != nullptr || fuse.act != 0;
+  p.splits = fused ? 1 : choose_splits(Mo, No, R);   // the fused epilogue needs the whole sum
+  p.bias = (const uint16_t*)fuse.bias; p.mask = (const uint16_t*)fuse.mask;
+  p.ldmask = fuse.ldmask; p.act = fuse.act; p.clip = fuse.clip;
   p.out = (uint16_t*)out; p.ldo = ldo;
   p.ws = (float*)workspace; p.ws_ld = ws_ld_for(No);
   p.flag = flag;
@@ -825,6 +873,46 @@ int mp_linear_bwd_wgrad_static(const void* X16, int64_t ldx, const void* dY16, i
 }
 
 size_t mp_static_scratch_bytes(void) { return (size_t)MP_STATIC_SCRATCH_FLOATS * sizeof(float); }
+
+// ---- layers with bias and activation ----------------------------------------------------------
+static int check_act(const char* name, int act, float clip) {
+  if (act != MP_ACT_NONE && act != MP_ACT_RELU && act != MP_ACT_CLIPPED_RELU)
+    return mp::set_error(MP_ERR_INVALID_ARG, "%s: unknown activation %d", name, act);
+  if (act == MP_ACT_CLIPPED_RELU && !(clip > 0.0f))
+    return mp::set_error(MP_ERR_INVALID_ARG, "%s: clip must be positive", name);
+  return MP_OK;
+}
+
+int mp_linear_fwd_act(const void* X16, int64_t ldx, const void* W16, int64_t ldw, const void* bias16,
+                      void* Y16, int64_t ldy, int64_t M, int64_t K, int64_t N, int act, float clip,
+                      void* workspace, size_t workspace_bytes, void* stream) {
+  if (int rc = check_act("mp_linear_fwd_act", act, clip)) return rc;
+  if (bias16 && !mp::aligned16(bias16))
+    return mp::set_error(MP_ERR_ALIGNMENT, "mp_linear_fwd_act: bias must be 16-byte aligned");
+  const Operand A{X16, ldx, false, M, K};
+  const Operand B{W16, ldw, true, N, K};
+  Fuse f;
+  f.bias = bias16; f.act = act; f.clip = clip;
+  return run_gemm("mp_linear_fwd_act", A, B, Y16, ldy, nullptr, false, workspace, workspace_bytes,
+                  (cudaStream_t)stream, f);
+}
+
+int mp_linear_bwd_dgrad_act(const void* dY16, int64_t lddy, const void* W16, int64_t ldw,
+                            const void* A16, int64_t lda, void* dX16, int64_t lddx, int64_t M,
+                            int64_t K, int64_t N, int act, float clip, void* workspace,
+                            size_t workspace_bytes, void* stream) {
+  if (int rc = check_act("mp_linear_bwd_dgrad_act", act, clip)) return rc;
+  if (act != MP_ACT_NONE) {
+    if (!A16) return mp::set_error(MP_ERR_INVALID_ARG, "mp_linear_bwd_dgrad_act: null layer input");
+    if (lda < K) return mp::set_error(MP_ERR_INVALID_ARG, "mp_linear_bwd_dgrad_act: lda < K");
+  }
+  const Operand A{dY16, lddy, false, M, N};
+  const Operand B{W16, ldw, false, K, N};
+  Fuse f;
+  f.mask = act != MP_ACT_NONE ? A16 : nullptr; f.ldmask = lda; f.act = act; f.clip = clip;
+  return run_gemm("mp_linear_bwd_dgrad_act", A, B, dX16, lddx, nullptr, false, workspace,
+                  workspace_bytes, (cudaStream_t)stream, f);
+}
 
 // Synchronises the device and returns the first device-side error recorded by a GEMM kernel
 // (MP_OK if none), clearing it.

@@ -303,6 +303,62 @@ mp_scale_upstream_kernel(const float* __restrict__ g32, uint16_t* __restrict__ o
   }
 }
 
+// Bias gradient, stage 1: FP32 column sums of dY over a slab of rows.  A block owns 64 columns
+// (one half2 per lane) and one slab; its 8 warps stride over the slab's rows, then add their
+// sums in warp order through shared memory.  partial[slab][n] is written once, no atomics.
+constexpr int kBiasSlabs = 64;
+__global__ void __launch_bounds__(kThreads)
+mp_bias_grad_partial_kernel(const uint16_t* __restrict__ dY, int64_t lddy, int64_t M, int64_t N,
+                            float* __restrict__ partial, int slabs) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int64_t col = (int64_t)blockIdx.x * 64 + lane * 2;
+  const int slab = blockIdx.y;
+  const int64_t rows_per = (M + slabs - 1) / slabs;
+  const int64_t r0 = slab * rows_per, r1 = r0 + rows_per < M ? r0 + rows_per : M;
+  float a0 = 0.0f, a1 = 0.0f;
+  if (col < N) {
+    const bool two = col + 1 < N;
+    for (int64_t r = r0 + warp; r < r1; r += 8) {
+      const uint16_t* src = dY + r * lddy + col;
+      if (two) {
+        const uint32_t w = *reinterpret_cast<const uint32_t*>(src);
+        a0 = __fadd_rn(a0, half_bits_to_float((uint16_t)(w & 0xFFFFu)));
+        a1 = __fadd_rn(a1, half_bits_to_float((uint16_t)(w >> 16)));
+      } else {
+        a0 = __fadd_rn(a0, half_bits_to_float(src[0]));
+      }
+    }
+  }
+  __shared__ float s0[8][32], s1[8][32];
+  s0[warp][lane] = a0;
+  s1[warp][lane] = a1;
+  __syncthreads();
+  if (warp == 0 && col < N) {
+    float t0 = s0[0][lane], t1 = s1[0][lane];
+#pragma unroll
+    for (int w = 1; w < 8; ++w) { t0 = __fadd_rn(t0, s0[w][lane]); t1 = __fadd_rn(t1, s1[w][lane]); }
+    partial[(int64_t)slab * N + col] = t0;
+    if (col + 1 < N) partial[(int64_t)slab * N + col + 1] = t1;
+  }
+}
+
+// Bias gradient, stage 2: add the slabs in ascending order, round to FP16, store, inspect.
+__global__ void __launch_bounds__(kThreads)
+mp_bias_grad_final_kernel(const float* __restrict__ partial, int slabs, int64_t N,
+                          uint16_t* __restrict__ db, mp_dev_state* st) {
+  const int64_t n = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+  uint32_t bad = 0;
+  if (n < N) {
+    float a = partial[n];
+    for (int s = 1; s < slabs; ++s) a = __fadd_rn(a, partial[(int64_t)s * N + n]);
+    const uint16_t h = float_to_half_bits(a);
+    db[n] = h;
+    bad = ((h & 0x7C00u) == 0x7C00u) ? 1u : 0u;
+  }
+  if (st != nullptr && __any_sync(0xFFFFFFFFu, bad != 0) && (threadIdx.x & 31) == 0)
+    atomicOr(&st->h.found_inf, 1);
+}
+
 // Loss-scale state machine, one thread (Section 3.1, item 1).
 __global__ void mp_loss_scale_update_kernel(mp_dev_state* st) {
   mp_state_host& h = st->h;
@@ -539,6 +595,38 @@ int mp_scale_upstream(const float* g32, void* dY16, int64_t n, const mp_state* s
   mp_scale_upstream_kernel<<<grid_for(blocks, sms, 16), kThreads, 0, (cudaStream_t)stream>>>(
       g32, (uint16_t*)dY16, n, state->dev);
   mp::count_launch();
+  MP_CUDA_TRY(cudaGetLastError());
+  return MP_OK;
+}
+
+static int bias_slabs(int64_t M) {
+  const int64_t want = (M + 255) / 256;
+  return (int)(want < 1 ? 1 : (want > kBiasSlabs ? kBiasSlabs : want));
+}
+
+size_t mp_bias_grad_workspace_bytes(int64_t M, int64_t N) {
+  if (M <= 0 || N <= 0) return 0;
+  return (size_t)bias_slabs(M) * (size_t)N * sizeof(float);
+}
+
+int mp_bias_grad(const void* dY16, int64_t lddy, void* db16, int64_t M, int64_t N, mp_state* state,
+                 void* workspace, size_t workspace_bytes, void* stream) {
+  if (!dY16 || !db16 || M <= 0 || N <= 0 || lddy < N)
+    return mp::set_error(MP_ERR_INVALID_ARG, "mp_bias_grad: bad argument");
+  if (!mp::aligned16(dY16) || !mp::aligned16(db16) || (lddy & 7) || (workspace && !mp::aligned16(workspace)))
+    return mp::set_error(MP_ERR_ALIGNMENT, "mp_bias_grad: buffers must be 16-byte aligned, lddy a multiple of 8");
+  const size_t need = mp_bias_grad_workspace_bytes(M, N);
+  if (!workspace || workspace_bytes < need)
+    return mp::set_error(MP_ERR_NOMEM, "mp_bias_grad: workspace of %zu bytes needed", need);
+  if (int rc = mp::check_device()) return rc;
+  const int slabs = bias_slabs(M);
+  cudaStream_t st = (cudaStream_t)stream;
+  const dim3 grid((unsigned)((N + 63) / 64), (unsigned)slabs);
+  mp_bias_grad_partial_kernel<<<grid, kThreads, 0, st>>>((const uint16_t*)dY16, lddy, M, N,
+                                                        (float*)workspace, slabs);
+  mp_bias_grad_final_kernel<<<(unsigned)((N + kThreads - 1) / kThreads), kThreads, 0, st>>>(
+      (const float*)workspace, slabs, N, (uint16_t*)db16, state ? state->dev : nullptr);
+  mp::count_launch(2);
   MP_CUDA_TRY(cudaGetLastError());
   return MP_OK;
 }

@@ -20,6 +20,7 @@ MP_ERR_CUDA, MP_ERR_TIMEOUT, MP_ERR_NOMEM, MP_ERR_TOO_LARGE = -4, -5, -6, -7
 MP_OPT_ADAM, MP_OPT_MOMENTUM = 0, 1
 MP_OP_FWD, MP_OP_DGRAD, MP_OP_WGRAD = 0, 1, 2
 MP_LOG_CAPACITY = 4096
+MP_ACT_NONE, MP_ACT_RELU, MP_ACT_CLIPPED_RELU = 0, 1, 2
 
 
 class MpError(RuntimeError):
@@ -58,6 +59,11 @@ SIGNATURES = {
     "mp_linear_bwd_wgrad": (_i32, [_p, _i64, _p, _i64, _p, _i64, _i64, _i64, _i64, _p, _p, _sz, _p]),
     "mp_linear_bwd_wgrad_static": (_i32, [_p, _i64, _p, _i64, _p, _i64, _i64, _i64, _i64, _p, _p]),
     "mp_static_scratch_bytes": (_sz, []),
+    "mp_linear_fwd_act": (_i32, [_p, _i64, _p, _i64, _p, _p, _i64, _i64, _i64, _i64, _i32, C.c_float, _p, _sz, _p]),
+    "mp_linear_bwd_dgrad_act": (_i32, [_p, _i64, _p, _i64, _p, _i64, _p, _i64, _i64, _i64, _i64, _i32,
+                                       C.c_float, _p, _sz, _p]),
+    "mp_bias_grad": (_i32, [_p, _i64, _p, _i64, _i64, _p, _p, _sz, _p]),
+    "mp_bias_grad_workspace_bytes": (_sz, [_i64, _i64]),
     "mp_master_update": (_i32, [_p, _p, C.POINTER(OptimConfig), _i32, _p]),
     "mp_loss_scale_update": (_i32, [_p, _p]),
     "mp_gemm_workspace_bytes": (_sz, [_i64, _i64, _i64, _i32]),
@@ -179,6 +185,43 @@ def mp_linear_bwd_wgrad_static(X16, dY16, dW16, state=None):
 
 def mp_static_scratch_bytes() -> int:
     return int(lib().mp_static_scratch_bytes())
+
+
+def mp_linear_fwd_act(X16, W16, bias16, Y16, act=MP_ACT_NONE, clip=20.0, workspace=None):
+    (x, ldx), (w, ldw), (y, ldy) = _mat(X16), _mat(W16), _mat(Y16)
+    M, K = X16.shape
+    N = W16.shape[1]
+    assert W16.shape[0] == K and tuple(Y16.shape) == (M, N)
+    b = None
+    if bias16 is not None:
+        assert bias16.numel() == N and bias16.is_contiguous()
+        b = _dev(bias16, torch.float16)
+    ws, nb = _ws(workspace)
+    _check(lib().mp_linear_fwd_act(x, ldx, w, ldw, b, y, ldy, M, K, N, act, clip, ws, nb, _stream()))
+
+
+def mp_linear_bwd_dgrad_act(dY16, W16, A16, dX16, act=MP_ACT_NONE, clip=20.0, workspace=None):
+    (dy, lddy), (w, ldw), (dx, lddx) = _mat(dY16), _mat(W16), _mat(dX16)
+    M, N = dY16.shape
+    K = W16.shape[0]
+    assert W16.shape[1] == N and tuple(dX16.shape) == (M, K)
+    a, lda = (None, 0) if A16 is None else _mat(A16)
+    ws, nb = _ws(workspace)
+    _check(lib().mp_linear_bwd_dgrad_act(dy, lddy, w, ldw, a, lda, dx, lddx, M, K, N, act, clip, ws, nb,
+                                         _stream()))
+
+
+def mp_bias_grad_workspace_bytes(M: int, N: int) -> int:
+    return int(lib().mp_bias_grad_workspace_bytes(M, N))
+
+
+def mp_bias_grad(dY16, db16, state=None, workspace=None):
+    dy, lddy = _mat(dY16)
+    M, N = dY16.shape
+    assert db16.numel() == N and db16.is_contiguous()
+    ws, nb = _ws(workspace)
+    _check(lib().mp_bias_grad(dy, lddy, _dev(db16, torch.float16), M, N,
+                              state.handle if state is not None else None, ws, nb, _stream()))
 
 
 def mp_master_update(plan, state, opt: OptimConfig, check_mode: int = 0):

@@ -1,0 +1,124 @@
+"""Parity of the bias / activation epilogues and of the bias gradient against the oracle."""
+import numpy as np
+import pytest
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+ACTS = {"none": 0, "relu": 1, "clipped_relu": 2}
+
+
+def _pad8(n):
+    return (n + 7) // 8 * 8
+
+
+def _h(x):
+    return np.ascontiguousarray(x, np.float32).astype(np.float16).view(np.uint16)
+
+
+def _dev(bits):
+    if bits.ndim == 1:
+        return torch.from_numpy(bits.view(np.float16).copy()).cuda()
+    r, c = bits.shape
+    buf = torch.zeros(r, _pad8(c), dtype=torch.float16, device="cuda")
+    buf[:, :c] = torch.from_numpy(bits.view(np.float16)).cuda()
+    return buf[:, :c]
+
+
+def _out(r, c):
+    return torch.full((r, _pad8(c)), 7.0, dtype=torch.float16, device="cuda")[:, :c]
+
+
+def _bits(t):
+    return t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+SHAPES = [(37, 64, 29), (300, 200, 520), (128, 72, 257), (129, 328, 264), (1, 8, 8)]
+
+
+@pytest.mark.parametrize("act", ["none", "relu", "clipped_relu"])
+@pytest.mark.parametrize("M,K,N", SHAPES)
+def test_fwd_bias_activation_integer_exact(orc, mp, act, M, K, N):
+    """Small-integer operands and bias: the FP32 value before the activation is exact, so the
+    GPU must match the oracle bit for bit."""
+    rng = np.random.default_rng(M + K + N)
+    X, W = _h(rng.integers(-2, 3, (M, K))), _h(rng.integers(-2, 3, (K, N)))
+    b = _h(rng.integers(-30, 31, N))
+    Y = _out(M, N)
+    ws = torch.empty(max(mp.mp_gemm_workspace_bytes(M, K, N, 0), 16), dtype=torch.uint8, device="cuda")
+    mp.mp_linear_fwd_act(_dev(X), _dev(W), _dev(b), Y, ACTS[act], 20.0, ws)
+    torch.cuda.synchronize()
+    assert mp.mp_gemm_device_status() == 0
+    want = orc.linear_fwd_act(X, W, b, act, clip=20.0)
+    assert (_bits(Y) == want).all()
+    if act == "clipped_relu" and M * N > 1000:
+        f = want.view(np.float16).astype(np.float32)
+        assert f.max() <= 20.0 and (f == 20.0).any() and (f == 0).any()
+    # no bias: same call with NULL
+    mp.mp_linear_fwd_act(_dev(X), _dev(W), None, Y, ACTS[act], 20.0, ws)
+    assert (_bits(Y) == orc.linear_fwd_act(X, W, None, act, clip=20.0)).all()
+
+
+@pytest.mark.parametrize("act", ["none", "relu", "clipped_relu"])
+@pytest.mark.parametrize("M,K,N", SHAPES)
+def test_dgrad_activation_mask_integer_exact(orc, mp, act, M, K, N):
+    rng = np.random.default_rng(M * 3 + K + N)
+    dY, W = _h(rng.integers(-2, 3, (M, N))), _h(rng.integers(-2, 3, (K, N)))
+    A = _h(np.clip(rng.integers(-15, 30, (M, K)), 0, 20))           # an activated output: 0 .. 20
+    A[0, 0] = 0x8000                                                # -0 does not pass
+    dX = _out(M, K)
+    ws = torch.empty(max(mp.mp_gemm_workspace_bytes(M, K, N, 1), 16), dtype=torch.uint8, device="cuda")
+    mp.mp_linear_bwd_dgrad_act(_dev(dY), _dev(W), _dev(A), dX, ACTS[act], 20.0, ws)
+    torch.cuda.synchronize()
+    assert mp.mp_gemm_device_status() == 0
+    want = orc.linear_bwd_dgrad_act(dY, W, A, act, clip=20.0)
+    assert (_bits(dX) == want).all()
+    if act != "none":
+        assert (want == 0).mean() > 0.3
+
+
+def test_fwd_act_random_values_within_tolerance(orc, mp):
+    rng = np.random.default_rng(1)
+    M, K, N = 384, 520, 264
+    X, W = _h(rng.standard_normal((M, K))), _h(rng.standard_normal((K, N)) / 8)
+    b = _h(rng.standard_normal(N))
+    Y = _out(M, N)
+    ws = torch.empty(max(mp.mp_gemm_workspace_bytes(M, K, N, 0), 16), dtype=torch.uint8, device="cuda")
+    mp.mp_linear_fwd_act(_dev(X), _dev(W), _dev(b), Y, ACTS["relu"], 20.0, ws)
+    got = _bits(Y).view(np.float16).astype(np.float64)
+    ex, ab = orc.linear_exact("fwd", X, W)
+    z = ex + b.view(np.float16).astype(np.float64)[None, :]
+    want = np.maximum(z, 0)
+    tol = 2.0 ** -10 * np.abs(z) + K * 2.0 ** -24 * (ab + 4.0) + 2.0 ** -24
+    assert (np.abs(got - want) <= tol).all()
+    assert (_bits(Y) == orc.linear_fwd_act(X, W, b, "relu")).mean() > 0.98
+
+
+@pytest.mark.parametrize("M,N", [(1, 8), (257, 13), (5000, 1000), (8192, 4096), (25600, 29)])
+def test_bias_grad(orc, mp, M, N):
+    rng = np.random.default_rng(M + N)
+    dYi = rng.integers(-3, 4, (M, N))
+    dY = _h(dYi)
+    db = torch.zeros(_pad8(N), dtype=torch.float16, device="cuda")
+    ws = torch.empty(max(mp.mp_bias_grad_workspace_bytes(M, N), 16), dtype=torch.uint8, device="cuda")
+    st = mp.State()
+    mp.mp_bias_grad(_dev(dY), db[:N], st, ws)
+    got = _bits(db)
+    assert (got[:N] == _h(dYi.sum(axis=0))).all() and (got[N:] == 0).all()   # integer sums: bit exact
+    if M * N <= 5_000_000:
+        assert (got[:N] == orc.bias_grad(dY)).all()
+    assert st.read().found_inf == 0
+    # random values: FP32 sums in another order, one FP16 rounding
+    if M * N <= 5_000_000:
+        dYr = _h(rng.standard_normal((M, N)) * 4)
+        mp.mp_bias_grad(_dev(dYr), db[:N], st, ws)
+        g = _bits(db)[:N].view(np.float16).astype(np.float64)
+        f = dYr.view(np.float16).astype(np.float64)
+        want, ab = f.sum(axis=0), np.abs(f).sum(axis=0)
+        assert (np.abs(g - want) <= 2.0 ** -10 * np.abs(want) + M * 2.0 ** -24 * ab + 2.0 ** -24).all()
+        assert (_bits(db)[:N] == orc.bias_grad(dYr)).mean() > 0.97
+    # an inf in the column sum raises the flag
+    dY2 = dY.copy(); dY2[M - 1, N - 1] = 0x7C00
+    mp.mp_bias_grad(_dev(dY2), db[:N], st, ws)
+    assert _bits(db)[N - 1] == 0x7C00 and st.read().found_inf == 1
+    st.close()
