@@ -266,6 +266,13 @@ class Layer:
     m: np.ndarray               # Adam first moment, or the momentum buffer
     v: np.ndarray | None        # Adam second moment
     chained: bool = False       # input is the previous layer's output
+    act: str = "none"           # activation after this layer's product ("none" for a top layer)
+    clip: float = 20.0
+    b32: np.ndarray | None = None   # FP32 master bias [N] (None: no bias)
+    b16: np.ndarray | None = None
+    bm: np.ndarray | None = None
+    bv: np.ndarray | None = None
+    db: np.ndarray | None = None
     X: np.ndarray | None = None
     Y: np.ndarray | None = None
     dY: np.ndarray | None = None
@@ -273,10 +280,17 @@ class Layer:
     dW: np.ndarray | None = None
 
 
-def make_layer(w32: np.ndarray, kind: str, chained: bool) -> Layer:
+def make_layer(w32: np.ndarray, kind: str, chained: bool, act: str = "none", clip: float = 20.0,
+               b32: np.ndarray | None = None) -> Layer:
     w32 = np.ascontiguousarray(w32, np.float32).copy()
-    return Layer(w32=w32, w16=f2h(w32), m=np.zeros_like(w32),
-                 v=np.zeros_like(w32) if kind == "adam" else None, chained=chained)
+    ly = Layer(w32=w32, w16=f2h(w32), m=np.zeros_like(w32),
+               v=np.zeros_like(w32) if kind == "adam" else None, chained=chained, act=act, clip=clip)
+    if b32 is not None:
+        ly.b32 = np.ascontiguousarray(b32, np.float32).copy()
+        ly.b16 = f2h(ly.b32)
+        ly.bm = np.zeros_like(ly.b32)
+        ly.bv = np.zeros_like(ly.b32) if kind == "adam" else None
+    return ly
 
 
 @dataclass
@@ -301,23 +315,39 @@ def train_step(layers: list[Layer], xs: list, gs: list, scaler: Scaler, opt: Opt
     S = scaler.S
     for l, ly in enumerate(layers):                       # forward, Section 3.1
         ly.X = layers[l - 1].Y if ly.chained else xs[l]
-        ly.Y = linear_fwd(ly.X, ly.w16, nthreads)
+        if ly.act == "none" and ly.b16 is None:
+            ly.Y = linear_fwd(ly.X, ly.w16, nthreads)
+        else:
+            ly.Y = linear_fwd_act(ly.X, ly.w16, ly.b16, ly.act, ly.clip, nthreads)
     flag = 0
     for l in range(L - 1, -1, -1):                        # backward in FP16
         ly = layers[l]
         feeds_next = l + 1 < L and layers[l + 1].chained
+        assert feeds_next or ly.act == "none", "a top layer has no activation"
+        # dY is the gradient at this layer's pre-activation: the layer above has already
+        # masked it with this layer's activation derivative (taken from this layer's output)
         ly.dY = layers[l + 1].dX if feeds_next else scale_upstream(gs[l], S)
         ly.dW = linear_bwd_wgrad(ly.X, ly.dY, nthreads)
-        ly.dX = linear_bwd_dgrad(ly.dY, ly.w16, nthreads)
+        below = layers[l - 1] if ly.chained else None
+        if below is not None and below.act != "none":
+            ly.dX = linear_bwd_dgrad_act(ly.dY, ly.w16, ly.X, below.act, below.clip, nthreads)
+        else:
+            ly.dX = linear_bwd_dgrad(ly.dY, ly.w16, nthreads)
         flag |= found_inf(ly.dW)                          # inspection, Section 3.1 item 1
+        if ly.b16 is not None:
+            ly.db = bias_grad(ly.dY)
+            flag |= found_inf(ly.db)
     if not flag:                                          # Section 3.2
         t = scaler.t + 1
         for ly in layers:
-            if opt.kind == "adam":
-                adam_update(ly.dW, ly.w32, ly.m, ly.v, ly.w16, S, opt.lr, opt.beta1, opt.beta2,
-                            opt.eps, t, opt.weight_decay)
-            else:
-                momentum_update(ly.dW, ly.w32, ly.m, ly.w16, S, opt.lr, opt.momentum,
+            pairs = [(ly.dW, ly.w32, ly.m, ly.v, ly.w16)]
+            if ly.b16 is not None:
+                pairs.append((ly.db, ly.b32, ly.bm, ly.bv, ly.b16))
+            for g16, w32, m, v, w16 in pairs:
+                if opt.kind == "adam":
+                    adam_update(g16, w32, m, v, w16, S, opt.lr, opt.beta1, opt.beta2, opt.eps, t,
                                 opt.weight_decay)
+                else:
+                    momentum_update(g16, w32, m, w16, S, opt.lr, opt.momentum, opt.weight_decay)
     scaler.update(flag)                                   # scale for the next iteration
     return StepRecord(flag, S, scaler.S, scaler.good, scaler.t)

@@ -24,10 +24,17 @@ class LinearStack:
     def __init__(self, shapes, chained, optimizer="adam", lr=1e-3, beta1=0.9, beta2=0.999,
                  eps=1e-8, momentum=0.9, weight_decay=0.0, init_scale=65536.0,
                  growth_interval=1000, min_scale=1.0, max_scale=2.0 ** 24, dynamic=True,
-                 device="cuda"):
+                 device="cuda", acts=None, clip=20.0, bias=False):
+        """acts[l]: mp.MP_ACT_* after layer l's product (a layer whose output feeds no chained
+        layer must have MP_ACT_NONE); bias: every layer gets a bias vector."""
         self.shapes = [tuple(s) for s in shapes]
         self.chained = list(chained)
         self.L = len(shapes)
+        self.acts = list(acts) if acts is not None else [mp.MP_ACT_NONE] * self.L
+        self.clip, self.has_bias = float(clip), bool(bias)
+        for l in range(self.L):
+            feeds = l + 1 < self.L and self.chained[l + 1]
+            assert feeds or self.acts[l] == mp.MP_ACT_NONE, "a top layer has no activation"
         self.device = torch.device(device)
         self.opt = mp.OptimConfig(mp.MP_OPT_ADAM if optimizer == "adam" else mp.MP_OPT_MOMENTUM,
                                   lr, beta1, beta2, eps, momentum, weight_decay)
@@ -41,6 +48,10 @@ class LinearStack:
         for s in sizes:
             offs.append(total)
             total += _align(s)
+        boffs = []                                   # biases follow the weights in the same buffers
+        for _, _, n in self.shapes:
+            boffs.append(total)
+            total += _align(n) if self.has_bias else 0
         self.offsets, self.total = offs, total
         f16 = dict(dtype=torch.float16, device=self.device)
         f32 = dict(dtype=torch.float32, device=self.device)
@@ -55,6 +66,10 @@ class LinearStack:
         self.w32 = [view(self.w32_flat, l) for l in range(self.L)]
         self.m = [view(self.m_flat, l) for l in range(self.L)]
         self.v = [view(self.v_flat, l) for l in range(self.L)] if self.v_flat is not None else None
+        bview = lambda flat, l: flat[boffs[l]:boffs[l] + self.shapes[l][2]] if self.has_bias else None
+        self.b16 = [bview(self.w16_flat, l) for l in range(self.L)]
+        self.db = [bview(self.dw_flat, l) for l in range(self.L)]
+        self.b32 = [bview(self.w32_flat, l) for l in range(self.L)]
         # one plan over the whole flat range: padding columns hold zeros and stay zero
         self.plan = mp.UpdatePlan([self.dw_flat], [self.w32_flat], [self.m_flat],
                                   [self.v_flat] if self.v_flat is not None else None,
@@ -74,14 +89,19 @@ class LinearStack:
         for m, k, n in self.shapes:
             for op in (mp.MP_OP_FWD, mp.MP_OP_DGRAD, mp.MP_OP_WGRAD):
                 need = max(need, mp.mp_gemm_workspace_bytes(m, k, n, op))
+            if self.has_bias:
+                need = max(need, mp.mp_bias_grad_workspace_bytes(m, n))
         self.workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=self.device)
 
     # ---- data movement (no arithmetic) ----
-    def load_weights(self, l: int, w32: torch.Tensor, w16: torch.Tensor):
-        """Copies an FP32 master [K,N] and its FP16 working copy into the stack."""
+    def load_weights(self, l: int, w32: torch.Tensor, w16: torch.Tensor, b32=None, b16=None):
+        """Copies an FP32 master [K,N] and its FP16 working copy (and a bias pair) into the stack."""
         n = self.shapes[l][2]
         self.w32[l][:, :n].copy_(w32)
         self.w16[l][:, :n].copy_(w16)
+        if b32 is not None:
+            self.b32[l].copy_(b32)
+            self.b16[l].copy_(b16)
 
     def X(self, l): return self.x[l][:, :self.shapes[l][1]]
     def Y(self, l): return self.y[l][:, :self.shapes[l][2]]
@@ -171,8 +191,12 @@ class LinearStack:
         for l in range(self.L):
             if not self.chained[l]:
                 self.x[l] = xs[l]
-            self._call("fwd", mp.mp_linear_fwd, self.x[l][:, :self.shapes[l][1]], self.W16(l), self.Y(l),
-                       self.workspace)
+            if self.acts[l] == mp.MP_ACT_NONE and not self.has_bias:
+                self._call("fwd", mp.mp_linear_fwd, self.x[l][:, :self.shapes[l][1]], self.W16(l), self.Y(l),
+                           self.workspace)
+            else:
+                self._call("fwd", mp.mp_linear_fwd_act, self.x[l][:, :self.shapes[l][1]], self.W16(l),
+                           self.b16[l], self.Y(l), self.acts[l], self.clip, self.workspace)
         for l in range(self.L - 1, -1, -1):
             if not self.feeds_next(l):
                 n = self.shapes[l][2]
@@ -185,8 +209,15 @@ class LinearStack:
             X = self.x[l][:, :self.shapes[l][1]]
             self._call("wgrad", mp.mp_linear_bwd_wgrad, X, self.dY(l), self.dW(l), self.state,
                        self.workspace)
-            self._call("dgrad", mp.mp_linear_bwd_dgrad, self.dY(l), self.W16(l), self.dX(l),
-                       self.workspace)
+            if self.has_bias:
+                self._call("bgrad", mp.mp_bias_grad, self.dY(l), self.db[l], self.state, self.workspace)
+            below = self.acts[l - 1] if self.chained[l] else mp.MP_ACT_NONE
+            if below == mp.MP_ACT_NONE:
+                self._call("dgrad", mp.mp_linear_bwd_dgrad, self.dY(l), self.W16(l), self.dX(l),
+                           self.workspace)
+            else:       # the layer below is activated: mask with its stored output (= this layer's input)
+                self._call("dgrad", mp.mp_linear_bwd_dgrad_act, self.dY(l), self.W16(l), X, self.dX(l),
+                           below, self.clip, self.workspace)
         if self.grad_sync is not None:       # data parallel: sum the FP16 gradients over ranks,
             self.grad_sync(self.dw_flat)     # then inspect the reduced gradients in the update call
         self._call("update", mp.mp_master_update, self.plan, self.state, self.opt,

@@ -23,20 +23,27 @@ def _pad_dev(bits):
     return buf
 
 
-def build_both(orc, cfg, dynamic=True):
+ACT_NAMES = {0: "none", 1: "relu", 2: "clipped_relu"}
+
+
+def build_both(orc, cfg, dynamic=True, acts=None, bias=False, clip=20.0):
     from paper_1805_10387_b200.stack import LinearStack
     L = len(cfg.shapes)
     chained = [cfg.chained(l) for l in range(L)]
+    acts = acts or [0] * L
     gpu = LinearStack(cfg.shapes, chained, optimizer=cfg.optimizer, lr=cfg.lr, beta1=cfg.beta1,
                       beta2=cfg.beta2, eps=cfg.eps, momentum=cfg.momentum,
-                      init_scale=cfg.init_scale, growth_interval=cfg.growth_interval, dynamic=dynamic)
+                      init_scale=cfg.init_scale, growth_interval=cfg.growth_interval, dynamic=dynamic,
+                      acts=acts, bias=bias, clip=clip)
     layers = []
     for l in range(L):
         w = synth.weights(cfg, l)
-        ly = orc.make_layer(w, cfg.optimizer, chained[l])
+        b = (synth.normal(cfg.seed, 9000 + l, cfg.shapes[l][2]) * 0.1).astype(np.float32) if bias else None
+        ly = orc.make_layer(w, cfg.optimizer, chained[l], ACT_NAMES[acts[l]], clip, b)
         layers.append(ly)
-        gpu.load_weights(l, torch.from_numpy(w).cuda(),
-                         torch.from_numpy(synth.fp16_bits(w).view(np.float16).reshape(w.shape)).cuda())
+        h16 = lambda a: torch.from_numpy(synth.fp16_bits(a).view(np.float16).reshape(a.shape)).cuda()
+        gpu.load_weights(l, torch.from_numpy(w).cuda(), h16(w),
+                         torch.from_numpy(b).cuda() if bias else None, h16(b) if bias else None)
         assert (synth.fp16_bits(w).reshape(w.shape) == ly.w16).all()
     sc = orc.Scaler(cfg.init_scale, cfg.growth_interval, dynamic=dynamic)
     opt = orc.Optim(kind=cfg.optimizer, lr=cfg.lr, beta1=cfg.beta1, beta2=cfg.beta2, eps=cfg.eps,
@@ -44,7 +51,7 @@ def build_both(orc, cfg, dynamic=True):
     return gpu, layers, sc, opt
 
 
-def drift_ok(got_bits, want_bits, what):
+def drift_ok(got_bits, want_bits, what, frac=1.0):
     """Free-running comparison: the two sides see inputs that may already differ by an FP16
     rounding (chained layers, updated weights), so the error is measured against the size of
     the tensor, not of each element."""
@@ -54,7 +61,10 @@ def drift_ok(got_bits, want_bits, what):
     if fin.any():
         rms = np.sqrt((w[fin] ** 2).mean())
         err = np.abs(g[fin] - w[fin])
-        assert (err <= 1e-2 * np.abs(w[fin]) + 2e-2 * rms + 2.0 ** -24).all(), (what, err.max(), rms)
+        ok = err <= 1e-2 * np.abs(w[fin]) + 2e-2 * rms + 2.0 ** -24
+        # with activations a value next to zero can fall on either side of the mask in the two
+        # free-running copies, which moves a few elements by more than a rounding
+        assert ok.mean() >= frac, (what, err.max(), rms, ok.mean())
 
 
 def forced_ok(orc, op, A_bits, B_bits, got_bits, what):
@@ -78,8 +88,9 @@ def forced_ok(orc, op, A_bits, B_bits, got_bits, what):
             assert (np.abs(g[big] - w[big]) / np.abs(w[big])).max() <= 1e-2, what
 
 
-def run_config(orc, mp, cfg, steps, dynamic=True):
-    gpu, layers, sc, opt = build_both(orc, cfg, dynamic)
+def run_config(orc, mp, cfg, steps, dynamic=True, acts=None, bias=False, clip=20.0):
+    gpu, layers, sc, opt = build_both(orc, cfg, dynamic, acts, bias, clip)
+    acts = acts or [0] * len(cfg.shapes)
     L = len(cfg.shapes)
     records = []
     for step in range(steps):
@@ -92,6 +103,7 @@ def run_config(orc, mp, cfg, steps, dynamic=True):
                 None if gpu.v is None else gpu.v[l][:, :cfg.shapes[l][2]].cpu().numpy().copy())
                for l in range(L)]
         w16_pre = [_bits(gpu.W16(l)) for l in range(L)]
+        b16_pre = [_bits(gpu.b16[l]) if bias else None for l in range(L)]
         t_pre = gpu.state.read().t
         gpu.step(dxs, dgs)
         rec = orc.train_step(layers, xs, gs, sc, opt)
@@ -107,14 +119,39 @@ def run_config(orc, mp, cfg, steps, dynamic=True):
         for l in range(L):
             Xg, Yg, dYg = _bits(gpu.X(l)), _bits(gpu.Y(l)), _bits(gpu.dY(l))
             dXg, dWg = _bits(gpu.dX(l)), _bits(gpu.dW(l))
-            forced_ok(orc, "fwd", Xg, w16_pre[l], Yg, f"Y{l} step {step}")
+            if acts[l] == 0 and not bias:
+                forced_ok(orc, "fwd", Xg, w16_pre[l], Yg, f"Y{l} step {step}")
+            else:       # the oracle's activated product of the operands the GPU read
+                want = orc.linear_fwd_act(np.ascontiguousarray(Xg), np.ascontiguousarray(w16_pre[l]),
+                                          np.ascontiguousarray(b16_pre[l]) if bias else None,
+                                          ACT_NAMES[acts[l]], clip)
+                wf, gf = _f(want), _f(Yg)
+                assert (np.abs(gf - wf) <= 2.0 ** -9 * np.abs(wf) + 2e-3 * np.sqrt((wf * wf).mean()) + 1e-6).all()
+                assert (Yg == want).mean() > 0.97
             forced_ok(orc, "wgrad", Xg, dYg, dWg, f"dW{l} step {step}")
-            forced_ok(orc, "dgrad", dYg, w16_pre[l], dXg, f"dX{l} step {step}")
+            below = acts[l - 1] if cfg.chained(l) else 0
+            if below == 0:
+                forced_ok(orc, "dgrad", dYg, w16_pre[l], dXg, f"dX{l} step {step}")
+            else:
+                want = orc.linear_bwd_dgrad_act(np.ascontiguousarray(dYg), np.ascontiguousarray(w16_pre[l]),
+                                                np.ascontiguousarray(Xg), ACT_NAMES[below], clip)
+                assert ((dXg == 0) == (want == 0)).mean() > 0.999          # same mask
+                wf, gf = _f(want), _f(dXg)
+                fin = np.isfinite(wf) & np.isfinite(gf)
+                assert (np.abs(gf - wf)[fin] <= 2.0 ** -9 * np.abs(wf[fin]) + 2e-3 * np.sqrt((wf[fin] ** 2).mean()) + 1e-7).all()
+            if bias:
+                dbg = _bits(gpu.db[l])
+                want = orc.bias_grad(np.ascontiguousarray(dYg))
+                wf, gf = _f(want), _f(dbg)
+                fin = np.isfinite(wf)
+                assert (np.isfinite(gf) == fin).all()
+                assert (np.abs(gf - wf)[fin] <= 2.0 ** -9 * np.abs(wf[fin]) + 1e-3 * np.abs(_f(dYg)).sum(axis=0)[fin] * 2.0 ** -10 + 1e-7).all()
             if not cfg.feeds_next(l):              # upstream scaling: bitwise
                 assert (dYg == orc.scale_upstream(gs[l], rec.S_before)).all()
-            drift_ok(Yg, layers[l].Y, f"Y{l} step {step}")
-            drift_ok(dXg, layers[l].dX, f"dX{l} step {step}")
-            drift_ok(dWg, layers[l].dW, f"dW{l} step {step}")
+            frac = 1.0 if not any(acts) else 0.98
+            drift_ok(Yg, layers[l].Y, f"Y{l} step {step}", frac)
+            drift_ok(dXg, layers[l].dX, f"dX{l} step {step}", frac)
+            drift_ok(dWg, layers[l].dW, f"dW{l} step {step}", frac)
             w_gpu = gpu.W32(l).cpu().numpy()
             if rec.found_inf:                       # skipped: bitwise unchanged
                 assert (w_gpu.view(np.uint32) == pre[l][0].view(np.uint32)).all()
@@ -215,3 +252,18 @@ def test_graph_replay_equals_call_by_call(orc, mp):
         assert torch.equal(fa.view(torch.int32), fb.view(torch.int32))
     assert torch.equal(a.w16_flat.view(torch.int16), b.w16_flat.view(torch.int16))
     a.close(); b.close()
+
+
+@pytest.mark.parametrize("name,shapes,acts,clip", [
+    ("c3", [(384, 136, 520), (384, 520, 136), (384, 136, 136)], [1, 0, 0], 20.0),       # ReLU inside the FFN pair
+    ("c4", [(512, 200, 200)] * 3 + [(512, 200, 29)], [2, 2, 2, 0], 20.0),              # clipped ReLU chain
+])
+def test_layers_with_bias_and_activation(orc, mp, name, shapes, acts, clip):
+    """The scaled-down recipes as real layers: bias on every layer, ReLU between the FFN pair,
+    clipped ReLU through the dense chain, bias gradients inspected and updated with the weights."""
+    cfg = synth.config(name)
+    cfg.shapes = shapes
+    cfg.chain = cfg.chain[:len(shapes)]
+    cfg.growth_interval = 2
+    recs = run_config(orc, mp, cfg, 4, acts=acts, bias=True, clip=clip)
+    assert len(recs) == 4

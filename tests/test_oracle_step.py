@@ -124,3 +124,51 @@ def test_natural_overflow_halves_until_it_fits(orc):
         else:
             seen_clean = True
     assert seen_clean and sc.skipped >= 2
+
+
+def test_relu_stack_equals_plain_stack_when_nothing_is_clipped(orc):
+    """If every pre-activation is positive and no bias is present, a ReLU stack is the plain
+    stack: outputs, gradients and updated state agree bit for bit; with biases of zero too."""
+    rng = np.random.default_rng(12)
+    M, K = 16, 24
+    w = [np.abs(rng.standard_normal((K, K))).astype(np.float32) / K for _ in range(3)]
+    x = synth.fp16_bits(np.abs(rng.standard_normal((M, K))).astype(np.float32))
+    g = (rng.standard_normal((M, K)) * 0.01).astype(np.float32)
+
+    def run(acts, bias):
+        layers = [orc.make_layer(w[l], "adam", l > 0, acts[l], 20.0,
+                                 np.zeros(K, np.float32) if bias else None) for l in range(3)]
+        sc = orc.Scaler(256.0, 100)
+        rec = orc.train_step(layers, [x, None, None], [None, None, g], sc, orc.Optim())
+        return layers, rec
+    plain, r0 = run(["none"] * 3, False)
+    relu, r1 = run(["relu", "relu", "none"], False)
+    relub, r2 = run(["relu", "clipped_relu", "none"], True)
+    assert r0.found_inf == r1.found_inf == r2.found_inf == 0
+    for a, b, c in zip(plain, relu, relub):
+        for name in ("Y", "dY", "dX", "dW", "w32", "w16"):
+            assert (getattr(a, name).view(np.uint8) == getattr(b, name).view(np.uint8)).all(), name
+            assert (getattr(a, name).view(np.uint8) == getattr(c, name).view(np.uint8)).all(), name
+    # the bias gradient is the column sum of the gradient at the pre-activation
+    for ly in relub:
+        assert (ly.db == orc.bias_grad(ly.dY)).all() and (ly.b16 == orc.f2h(ly.b32)).all()
+        assert (ly.b32 != 0).any()                       # Adam moved the biases
+
+
+def test_activation_gradient_is_taken_from_the_stored_output(orc):
+    """Two-layer ReLU stack: rows of the hidden output that are zero get no gradient through
+    the first layer, whatever the upstream gradient."""
+    rng = np.random.default_rng(13)
+    M, K = 12, 16
+    w0 = rng.standard_normal((K, K)).astype(np.float32) / 4
+    w1 = rng.standard_normal((K, K)).astype(np.float32) / 4
+    layers = [orc.make_layer(w0, "adam", False, "relu"), orc.make_layer(w1, "adam", True, "none")]
+    x = synth.fp16_bits(rng.standard_normal((M, K)).astype(np.float32))
+    g = rng.standard_normal((M, K)).astype(np.float32)
+    w1_used = layers[1].w16.copy()                     # the step rewrites the working copy
+    orc.train_step(layers, [x, None], [None, g], orc.Scaler(4.0, 100), orc.Optim())
+    hidden = layers[0].Y.view(np.float16).astype(np.float32)
+    assert (hidden >= 0).all() and (hidden == 0).any() and (hidden > 0).any()
+    assert (layers[0].dY[hidden == 0] == 0).all()
+    full = orc.linear_bwd_dgrad(layers[1].dY, w1_used)
+    assert (layers[0].dY[hidden > 0] == full[hidden > 0]).all()
