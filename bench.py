@@ -129,7 +129,13 @@ def run_reference(args):
     from paper_1805_10387_b200 import synth
     orc.build()
     cfg = synth.config("c2" if args.workload == "c5" else args.workload)
-    rows, upd = 48, 1 << 20
+    # size the per-step sample so that the whole run (warm-up + steps) takes about two minutes
+    upd = 1 << 20
+    data = None
+    dt, _, _, data = oracle_sample_step(orc, synth, cfg, 8, upd, data)
+    dt, _, _, data = oracle_sample_step(orc, synth, cfg, 8, upd, data)
+    budget = 120.0 / max(1, args.steps + args.warmup)
+    rows = int(max(4, min(64, 8 * budget / max(dt, 1e-3))))
     data = None
     for _ in range(args.warmup):
         _, _, _, data = oracle_sample_step(orc, synth, cfg, rows, upd, data)

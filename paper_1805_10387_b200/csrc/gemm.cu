@@ -1,12 +1,17 @@
-// FP16-in / FP32-accumulate matrix products of the step (Section 3.1 of the paper) as one
-// persistent, warp-specialised tcgen05 kernel for sm_100a:
+// FP16-in / FP32-accumulate matrix products of the step (Section 3.1 of the paper) as persistent,
+// warp-specialised tcgen05 kernels for sm_100a.  Both kernels share one pipeline:
 //
-//   warp 0      TMA producer: tensor-map loads into a 4-stage shared-memory ring
-//   warp 1      MMA issuer: tcgen05.mma (128x256x16, FP16 x FP16 -> FP32) into tensor memory;
-//               owns the TMEM allocation (two 256-column accumulators, so the epilogue of one
-//               tile overlaps the main loop of the next)
-//   warps 2-5   epilogue: tcgen05.ld, round to FP16 (nearest even, overflow to inf), store;
-//               for the weight gradient also the inf/NaN inspection of what is stored
+//   warp 0      TMA producer: tensor-map loads into a shared-memory ring (128-byte swizzle)
+//   warp 1      MMA issuer: tcgen05.mma (FP16 x FP16 -> FP32) into tensor memory; owns the TMEM
+//               allocation (two 256-column accumulators, so the epilogue of one tile overlaps
+//               the main loop of the next)
+//   warps 2-5   epilogue: tcgen05.ld, optional bias / activation / mask, round to FP16 (nearest
+//               even, overflow to inf), store; for the weight gradient also the inf/NaN
+//               inspection of what is stored
+//
+//   mp_gemm_pair_kernel  clusters of two CTAs, tcgen05.mma.cta_group::2, one 256 x 256 tile per
+//                        pair, 6 stages x 32 KiB per CTA; used for outputs of more than 128 rows
+//   mp_gemm_kernel       one CTA per 128 x 256 tile, cta_group::1, 4 stages x 48 KiB
 //
 // The three products differ only in which operand dimension is contiguous in memory:
 //   forward   Y  = X  * W      A = X  (reduction contiguous)   B = W  (output dim contiguous)
