@@ -175,6 +175,8 @@ def run_update_sweep(args):
     sampler.start()
     launches0 = mp.mp_kernel_launch_count()
     for P, n in ((1_000_000, 1), (10_000_000, 8), (100_000_000, 64), (1_000_000_000, 500)):
+        if P > args.max_params:
+            break
         counts = synth.tensor_sizes(P, n, 4)
         offs, tot = [], 0
         for c in counts:
@@ -248,6 +250,7 @@ def main():
     ap.add_argument("--workload", default="c2", choices=["c2", "c3", "c4", "c5"])
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--max-params", type=float, default=1e9, help="c5: largest parameter count of the sweep")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
