@@ -13,6 +13,9 @@
 struct mp_dev_state {
   mp_state_host h;
   int64_t log_count;  // records ever written; slot = log_count % MP_LOG_CAPACITY
+  // Work distribution of the fused update: next chunk to hand out, and blocks that have finished.
+  // Both are zero between launches (the last block to finish clears them).
+  unsigned int update_ticket, update_done;
   mp_log_record log[MP_LOG_CAPACITY];
 };
 

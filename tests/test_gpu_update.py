@@ -96,7 +96,7 @@ def test_check_finite_exhaustive_patterns(orc, mp):
 
 
 @pytest.mark.parametrize("kind", ["adam", "momentum"])
-@pytest.mark.parametrize("counts", [[1], [5, 0, 13, 4096, 4097, 8191, 3, 100000], [1 << 20]])
+@pytest.mark.parametrize("counts", [[1], [5, 0, 13, 4096, 4097, 8191, 8192, 8193, 3, 100000], [1 << 20]])
 def test_master_update_matches_oracle(orc, mp, kind, counts):
     rng = np.random.default_rng(len(counts))
     adam = kind == "adam"
@@ -160,7 +160,7 @@ def test_master_update_matches_oracle(orc, mp, kind, counts):
 
 
 def test_overflow_step_is_a_bitwise_no_op(orc, mp):
-    counts = [777, 4096 * 3 + 5]
+    counts = [777, 8192 * 3 + 5]
     T = Tensors(counts)
     rng = np.random.default_rng(3)
     for flat in (T.w32, T.m, T.v):
@@ -168,7 +168,7 @@ def test_overflow_step_is_a_bitwise_no_op(orc, mp):
     T.v.abs_()
     T.w16.copy_(T.w32.half())
     T.g16.copy_(torch.from_numpy(rng.standard_normal(T.g16.numel()).astype(np.float16)).cuda())
-    T.g16[T.offs[1] + 4096 * 3 + 4] = float("inf")            # in the ragged tail of the last chunk
+    T.g16[T.offs[1] + 8192 * 3 + 4] = float("inf")            # in the ragged tail of the last chunk
     before = [x.clone() for x in (T.w32, T.m, T.v, T.w16)]
     st = mp.State(init_scale=4.0)
     plan = T.plan(mp)
