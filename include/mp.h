@@ -193,6 +193,23 @@ int mp_bias_grad(const void* dY16, int64_t lddy, void* db16, int64_t M, int64_t 
                  void* workspace, size_t workspace_bytes, void* stream);
 size_t mp_bias_grad_workspace_bytes(int64_t M, int64_t N);
 
+/* LSTM cell for a gate product G = [x;h] W of 4H columns in the order i, f, g, o (the GNMT-like
+ * layers of Section 5; the paper gives no arithmetic, so: FP16 gates and states in memory, the
+ * cell evaluated in FP32 with sigma(x) = 1/(1+exp(-x)) and tanh, one rounding per output).
+ *   c_new = sigma(f) c_prev + sigma(i) tanh(g),   h = sigma(o) tanh(c_new)
+ * G16 [M,4H] with ldg >= 4H; c_prev16, c_new16, h16 dense [M,H]; H and ldg multiples of 8. */
+int mp_lstm_cell_fwd(const void* G16, int64_t ldg, const void* c_prev16, void* c_new16, void* h16,
+                     int64_t M, int64_t H, void* stream);
+
+/* Backward of the cell from the stored FP16 gates and states: dh16 is the gradient at h,
+ * dc_in16 the gradient arriving at c_new from the next time step (NULL = none).  Writes dG16
+ * [M,4H] (gradient at the gate pre-activations, the dY of the gate product's backward calls)
+ * and dc_prev16 [M,H]; tanh(c_new) is taken from the stored FP16 c_new.  Gradients stay
+ * multiplied by the loss scale. */
+int mp_lstm_cell_bwd(const void* G16, int64_t ldg, const void* c_prev16, const void* c_new16,
+                     const void* dh16, const void* dc_in16, void* dG16, int64_t lddg, void* dc_prev16,
+                     int64_t M, int64_t H, void* stream);
+
 /* ---- auxiliaries --------------------------------------------------------------------- */
 
 enum { MP_OP_FWD = 0, MP_OP_DGRAD = 1, MP_OP_WGRAD = 2 };

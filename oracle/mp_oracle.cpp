@@ -266,6 +266,49 @@ void orc_bias_grad(const uint16_t* dY, int64_t lddy, uint16_t* db, int64_t M, in
   }
 }
 
+// ------------------------------------------------------------------ LSTM cell
+// The GNMT-like models of Section 5 feed their gate product [x;h] W (four gates of H columns
+// each, order i, f, g, o) to an LSTM cell.  Reading (the paper states no arithmetic): gates and
+// states are stored FP16, the cell is evaluated in FP32 from those FP16 values with
+// sigma(x) = 1 / (1 + exp(-x)) and tanh, and each output is rounded to FP16 once.
+static inline float sigm(float x) { return 1.0f / (1.0f + std::exp(-x)); }
+
+// c_new = sigma(f) c_prev + sigma(i) tanh(g);  h = sigma(o) tanh(c_new)
+void orc_lstm_cell_fwd(const uint16_t* G, int64_t ldg, const uint16_t* c_prev, uint16_t* c_new,
+                       uint16_t* h, int64_t M, int64_t H) {
+  for (int64_t m = 0; m < M; ++m)
+    for (int64_t j = 0; j < H; ++j) {
+      const float i = sigm(h2f(G[m * ldg + j])), f = sigm(h2f(G[m * ldg + H + j]));
+      const float g = std::tanh(h2f(G[m * ldg + 2 * H + j])), o = sigm(h2f(G[m * ldg + 3 * H + j]));
+      const float c = f * h2f(c_prev[m * H + j]) + i * g;
+      c_new[m * H + j] = f2h(c);
+      h[m * H + j] = f2h(o * std::tanh(c));
+    }
+}
+
+// Backward of the cell from the stored FP16 gates and states.  dh: gradient at h; dc_in:
+// gradient arriving at c_new from the next time step (may be null = 0).  tanh(c_new) is taken
+// from the stored FP16 c_new.  Writes dG [M,4H] (gradient at the gate pre-activations) and
+// dc_prev, all FP16, still multiplied by the loss scale.
+void orc_lstm_cell_bwd(const uint16_t* G, int64_t ldg, const uint16_t* c_prev,
+                       const uint16_t* c_new, const uint16_t* dh, const uint16_t* dc_in,
+                       uint16_t* dG, int64_t lddg, uint16_t* dc_prev, int64_t M, int64_t H) {
+  for (int64_t m = 0; m < M; ++m)
+    for (int64_t j = 0; j < H; ++j) {
+      const float i = sigm(h2f(G[m * ldg + j])), f = sigm(h2f(G[m * ldg + H + j]));
+      const float g = std::tanh(h2f(G[m * ldg + 2 * H + j])), o = sigm(h2f(G[m * ldg + 3 * H + j]));
+      const float tc = std::tanh(h2f(c_new[m * H + j]));
+      const float dhv = h2f(dh[m * H + j]);
+      float dc = dhv * o * (1.0f - tc * tc);
+      if (dc_in) dc = dc + h2f(dc_in[m * H + j]);
+      dG[m * lddg + j] = f2h(dc * g * (i * (1.0f - i)));
+      dG[m * lddg + H + j] = f2h(dc * h2f(c_prev[m * H + j]) * (f * (1.0f - f)));
+      dG[m * lddg + 2 * H + j] = f2h(dc * i * (1.0f - g * g));
+      dG[m * lddg + 3 * H + j] = f2h(dhv * tc * (o * (1.0f - o)));
+      dc_prev[m * H + j] = f2h(dc * f);
+    }
+}
+
 // ----------------------------------------------------- upstream scaling (O3)
 // Section 3.1 item 1: the loss (here: the gradient entering the top layer) is
 // multiplied by the current scale S, in FP32, then stored as FP16.

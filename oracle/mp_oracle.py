@@ -60,6 +60,8 @@ def lib():
         L.orc_linear_fwd_act.argtypes = [p, i64, p, i64, p, p, i64, i64, i64, i64, i32, f32, i32]
         L.orc_linear_bwd_dgrad_act.argtypes = [p, i64, p, i64, p, i64, p, i64, i64, i64, i64, i32, f32, i32]
         L.orc_bias_grad.argtypes = [p, i64, p, i64, i64]
+        L.orc_lstm_cell_fwd.argtypes = [p, i64, p, p, p, i64, i64]
+        L.orc_lstm_cell_bwd.argtypes = [p, i64, p, p, p, p, p, i64, p, i64, i64]
         L.orc_scale_upstream.argtypes = [p, f32, p, i64]
         L.orc_found_inf.restype = i32; L.orc_found_inf.argtypes = [p, i64]
         L.orc_adam_update.argtypes = [p, p, p, p, p, i64, f32, f32, f32, f32, f32, f32, i64]
@@ -161,6 +163,26 @@ def bias_grad(dY16) -> np.ndarray:
     db = np.empty(N, np.uint16)
     lib().orc_bias_grad(_ptr(dY16), N, _ptr(db), M, N)
     return db
+
+
+def lstm_cell_fwd(G16, c_prev16):
+    """(c_new, h) of an LSTM cell from the FP16 gate pre-activations [M,4H] (order i,f,g,o)."""
+    _chk(G16, np.uint16); _chk(c_prev16, np.uint16)
+    M, H4 = G16.shape; H = H4 // 4; assert c_prev16.shape == (M, H)
+    c = np.empty((M, H), np.uint16); h = np.empty((M, H), np.uint16)
+    lib().orc_lstm_cell_fwd(_ptr(G16), H4, _ptr(c_prev16), _ptr(c), _ptr(h), M, H)
+    return c, h
+
+
+def lstm_cell_bwd(G16, c_prev16, c_new16, dh16, dc_in16=None):
+    """(dG [M,4H], dc_prev [M,H]) from the stored gates and states."""
+    for a in (G16, c_prev16, c_new16, dh16):
+        _chk(a, np.uint16)
+    M, H4 = G16.shape; H = H4 // 4
+    dG = np.empty((M, H4), np.uint16); dcp = np.empty((M, H), np.uint16)
+    lib().orc_lstm_cell_bwd(_ptr(G16), H4, _ptr(c_prev16), _ptr(c_new16), _ptr(dh16),
+                            _ptr(dc_in16) if dc_in16 is not None else None, _ptr(dG), H4, _ptr(dcp), M, H)
+    return dG, dcp
 
 
 _OPS = {"fwd": 0, "dgrad": 1, "wgrad": 2}

@@ -8,7 +8,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_PKG)
 CSRC = os.path.join(_PKG, "csrc")
 LIB = os.path.join(_PKG, "libmp_b200.so")
-SOURCES = ["update.cu", "gemm.cu"]
+SOURCES = ["update.cu", "gemm.cu", "lstm.cu"]
 HEADERS = ["common.h", "ptx.cuh", os.path.join(_ROOT, "include", "mp.h")]
 
 

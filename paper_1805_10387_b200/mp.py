@@ -64,6 +64,8 @@ SIGNATURES = {
                                        C.c_float, _p, _sz, _p]),
     "mp_bias_grad": (_i32, [_p, _i64, _p, _i64, _i64, _p, _p, _sz, _p]),
     "mp_bias_grad_workspace_bytes": (_sz, [_i64, _i64]),
+    "mp_lstm_cell_fwd": (_i32, [_p, _i64, _p, _p, _p, _i64, _i64, _p]),
+    "mp_lstm_cell_bwd": (_i32, [_p, _i64, _p, _p, _p, _p, _p, _i64, _p, _i64, _i64, _p]),
     "mp_master_update": (_i32, [_p, _p, C.POINTER(OptimConfig), _i32, _p]),
     "mp_loss_scale_update": (_i32, [_p, _p]),
     "mp_gemm_workspace_bytes": (_sz, [_i64, _i64, _i64, _i32]),
@@ -222,6 +224,26 @@ def mp_bias_grad(dY16, db16, state=None, workspace=None):
     ws, nb = _ws(workspace)
     _check(lib().mp_bias_grad(dy, lddy, _dev(db16, torch.float16), M, N,
                               state.handle if state is not None else None, ws, nb, _stream()))
+
+
+def mp_lstm_cell_fwd(G16, c_prev16, c_new16, h16):
+    g, ldg = _mat(G16)
+    M, H = c_prev16.shape
+    assert G16.shape == (M, 4 * H) and c_prev16.is_contiguous() and c_new16.is_contiguous() and h16.is_contiguous()
+    _check(lib().mp_lstm_cell_fwd(g, ldg, _dev(c_prev16, torch.float16), _dev(c_new16, torch.float16),
+                                  _dev(h16, torch.float16), M, H, _stream()))
+
+
+def mp_lstm_cell_bwd(G16, c_prev16, c_new16, dh16, dc_in16, dG16, dc_prev16):
+    g, ldg = _mat(G16)
+    dg, lddg = _mat(dG16)
+    M, H = c_prev16.shape
+    for t in (c_prev16, c_new16, dh16, dc_prev16):
+        assert t.is_contiguous() and tuple(t.shape) == (M, H)
+    _check(lib().mp_lstm_cell_bwd(g, ldg, _dev(c_prev16, torch.float16), _dev(c_new16, torch.float16),
+                                  _dev(dh16, torch.float16),
+                                  _dev(dc_in16, torch.float16) if dc_in16 is not None else None,
+                                  dg, lddg, _dev(dc_prev16, torch.float16), M, H, _stream()))
 
 
 def mp_master_update(plan, state, opt: OptimConfig, check_mode: int = 0):

@@ -122,3 +122,47 @@ def test_bias_grad(orc, mp, M, N):
     mp.mp_bias_grad(_dev(dY2), db[:N], st, ws)
     assert _bits(db)[N - 1] == 0x7C00 and st.read().found_inf == 1
     st.close()
+
+
+# ------------------------------------------------------------------ LSTM cell
+@pytest.mark.parametrize("M,H", [(1, 8), (37, 64), (640, 1024)])
+def test_lstm_cell_forward_and_backward(orc, mp, M, H):
+    """Elementwise cell kernels against the oracle: both evaluate sigma and tanh in FP32 from the
+    same FP16 inputs, with different exp/tanh routines, so results agree to one FP16 unit in
+    the last place and nearly all outputs are identical bits."""
+    rng = np.random.default_rng(M + H)
+    G = _h(rng.standard_normal((M, 4 * H)) * 2.5)
+    c = _h(rng.standard_normal((M, H)))
+    Gd = _dev(G)
+    cd = torch.from_numpy(c.view(np.float16).copy()).cuda()
+    cn = torch.empty(M, H, dtype=torch.float16, device="cuda"); h = torch.empty_like(cn)
+    mp.mp_lstm_cell_fwd(Gd, cd, cn, h)
+    wc, wh = orc.lstm_cell_fwd(G, c)
+
+    def close(got_bits, want_bits, frac=0.995, scale=None):
+        g = got_bits.view(np.float16).astype(np.float64); w = want_bits.view(np.float16).astype(np.float64)
+        fin = np.isfinite(w)
+        assert (np.isfinite(g) == fin).all()
+        tol = 2.0 ** -10 * np.abs(w) + 2.0 ** -24                                 # one FP16 ulp
+        if scale is not None:
+            # factors like 1 - sigma(x) cancel: an FP32 ulp of sigma is an absolute, not a
+            # relative, error of the factor, so allow 1e-5 of the incoming gradient's size
+            tol = tol + 1e-5 * np.tile(scale, (1, w.shape[1] // scale.shape[1]))
+        assert (np.abs(g - w)[fin] <= tol[fin]).all()
+        assert (got_bits == want_bits).mean() >= frac
+    close(_bits(cn), wc); close(_bits(h), wh)
+    # backward, fed with the oracle's stored c_new so that both sides see identical inputs
+    dh = _h(rng.standard_normal((M, H)) * 64); dci = _h(rng.standard_normal((M, H)) * 64)
+    dG = _out(M, 4 * H); dcp = torch.empty(M, H, dtype=torch.float16, device="cuda")
+    t16 = lambda b: torch.from_numpy(b.view(np.float16).copy()).cuda()
+    for dc_bits in (dci, None):
+        mp.mp_lstm_cell_bwd(Gd, cd, t16(wc), t16(dh), None if dc_bits is None else t16(dc_bits), dG, dcp)
+        wG, wcp = orc.lstm_cell_bwd(G, c, wc, dh, dc_bits)
+        sc = np.abs(dh.view(np.float16).astype(np.float64)) + \
+            (0 if dc_bits is None else np.abs(dc_bits.view(np.float16).astype(np.float64)))
+        close(_bits(dG), wG, 0.98, sc); close(_bits(dcp), wcp, 0.98, sc)
+    # saturated gates and an overflowing gradient behave like the oracle's (inf stays inf)
+    Gs = _h(np.full((M, 4 * H), 30.0)); dh2 = dh.copy(); dh2[0, 0] = 0x7C00
+    mp.mp_lstm_cell_bwd(_dev(Gs), cd, t16(wc), t16(dh2), None, dG, dcp)
+    wG, wcp = orc.lstm_cell_bwd(Gs, c, wc, dh2, None)
+    assert ((_bits(dG) & 0x7C00) == 0x7C00).sum() == ((wG & 0x7C00) == 0x7C00).sum()
