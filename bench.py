@@ -250,6 +250,8 @@ def main():
     ap.add_argument("--workload", default="c2", choices=["c2", "c3", "c4", "c5"])
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--real-layers", action="store_true",
+                    help="biases on every layer and an activation inside every chain (ReLU; clipped ReLU for c4)")
     ap.add_argument("--max-params", type=float, default=1e9, help="c5: largest parameter count of the sweep")
     args = ap.parse_args()
     if args.impl == "reference":
@@ -277,9 +279,13 @@ def main():
     cfg = synth.config(args.workload)
     L = len(cfg.shapes)
     chained = [cfg.chained(l) for l in range(L)]
+    acts = None
+    if args.real_layers:
+        act = mp.MP_ACT_CLIPPED_RELU if cfg.name == "c4" else mp.MP_ACT_RELU
+        acts = [act if (l + 1 < L and chained[l + 1]) else mp.MP_ACT_NONE for l in range(L)]
     stack = LinearStack(cfg.shapes, chained, optimizer=cfg.optimizer, lr=cfg.lr, beta1=cfg.beta1,
                         beta2=cfg.beta2, eps=cfg.eps, momentum=cfg.momentum, init_scale=cfg.init_scale,
-                        growth_interval=cfg.growth_interval)
+                        growth_interval=cfg.growth_interval, acts=acts, bias=args.real_layers)
     if world > 1:      # data parallel over rows: weights replicated, FP16 weight gradients summed
         from paper_1805_10387_b200 import dp
         stack.grad_sync = dp.allreduce_gradients
@@ -287,7 +293,11 @@ def main():
     gen.manual_seed(1234 + cfg.seed)           # same weights on every rank
     for l, (M, K, N) in enumerate(cfg.shapes):
         w = torch.randn(K, N, generator=gen, device="cuda") / K ** 0.5
-        stack.load_weights(l, w, w.half())
+        if args.real_layers:
+            b = torch.randn(N, generator=gen, device="cuda") * 0.1
+            stack.load_weights(l, w, w.half(), b, b.half())
+        else:
+            stack.load_weights(l, w, w.half())
     gen.manual_seed(99 + rank)                 # each rank its own rows
     xs, gs, xs_host, gs_host = [], [], [], []
     for l, (M, K, N) in enumerate(cfg.shapes):
@@ -399,6 +409,8 @@ def main():
         "config": {"workload": cfg.name + ": " + cfg.note, "layers": L, "params": cfg.n_params(),
                    "gemm_gflop_per_step": flops_step / 1e9, "optimizer": cfg.optimizer,
                    "parallelism": f"dp{world}" if world > 1 else "single",
+                   "layers_kind": "bias + activation (fused epilogues) + bias gradients" if args.real_layers
+                                  else "plain linear",
                    "cache": "per-step working set (weights, moments, activations) far exceeds the 126 MB L2"},
         "e2e": {"value": e2e_val, "unit": "TFLOP/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": ms_e2e / args.steps},

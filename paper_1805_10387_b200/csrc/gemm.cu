@@ -91,8 +91,48 @@ __device__ __forceinline__ void report_timeout(B* bars) {
 // (TMEM lane) and walks the columns in chunks of 32.  tmem_acc is the TMEM address of the
 // accumulator's first column in this warp's lane quarter.  Returns nonzero if an inf or NaN
 // was stored as FP16.
+// Activation mask of one thread's row of a tile, one bit per column (word c = columns
+// 32c .. 32c+31): 1 where the layer input (the activated FP16 output of the layer below)
+// lies strictly inside the activation's linear range.  Called BEFORE the thread waits for the
+// accumulator, so the global loads (a DRAM round trip each when the input has left L2) run
+// under the tile's main loop instead of stretching the epilogue.
+__device__ __forceinline__ void load_pass_bits(const GemmParams& p, int row, int n0, uint32_t (&bits)[BN / 32]) {
+  const bool row_ok = row < p.Mo;
+#pragma unroll 4
+  for (int c = 0; c < BN / 32; ++c) {
+    const int col0 = n0 + c * 32;
+    uint32_t b = 0;
+    if (row_ok && col0 < p.No) {
+      const uint16_t* mrow = p.mask + (int64_t)row * p.ldmask + col0;
+      uint32_t mw[16];
+      if (col0 + 32 <= p.No) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const uint4 q4 = __ldg(reinterpret_cast<const uint4*>(mrow) + j);
+          mw[4 * j] = q4.x; mw[4 * j + 1] = q4.y; mw[4 * j + 2] = q4.z; mw[4 * j + 3] = q4.w;
+        }
+      } else {
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          const uint32_t lo = (col0 + 2 * j < p.No) ? __ldg(mrow + 2 * j) : 0u;
+          const uint32_t hi = (col0 + 2 * j + 1 < p.No) ? __ldg(mrow + 2 * j + 1) : 0u;
+          mw[j] = lo | (hi << 16);
+        }
+      }
+#pragma unroll
+      for (int j = 0; j < 32; ++j) {
+        const uint16_t hm = (uint16_t)((j & 1) ? (mw[j >> 1] >> 16) : (mw[j >> 1] & 0xFFFFu));
+        const float y = __half2float(__ushort_as_half(hm));
+        const bool pass = p.act == 2 ? (y > 0.0f && y < p.clip) : (y > 0.0f);
+        b |= (pass ? 1u : 0u) << j;
+      }
+    }
+    bits[c] = b;
+  }
+}
+
 __device__ __forceinline__ uint32_t epilogue_tile(const GemmParams& p, uint32_t tmem_acc, int row,
-                                                  int n0, int split) {
+                                                  int n0, int split, const uint32_t* pass_bits = nullptr) {
   const bool row_ok = row < p.Mo;
   uint32_t bad = 0;
 #pragma unroll 1
@@ -117,13 +157,31 @@ __device__ __forceinline__ uint32_t epilogue_tile(const GemmParams& p, uint32_t 
         }
       }
     } else {
+      const bool full_chunk = col0 + 32 <= p.No;
       if (p.bias != nullptr || (p.act != 0 && p.mask == nullptr)) {
         // forward flavour, on the FP32 values: + bias, then the activation
+        uint32_t bw[16];                          // 32 bias values as packed halves (0 if absent)
+        if (p.bias != nullptr && full_chunk) {
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {           // same address in every thread: one broadcast load
+            const uint4 q4 = __ldg(reinterpret_cast<const uint4*>(p.bias + col0) + j);
+            bw[4 * j] = q4.x; bw[4 * j + 1] = q4.y; bw[4 * j + 2] = q4.z; bw[4 * j + 3] = q4.w;
+          }
+        } else {
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const uint32_t lo = (p.bias != nullptr && col0 + 2 * j < p.No) ? __ldg(p.bias + col0 + 2 * j) : 0u;
+            const uint32_t hi = (p.bias != nullptr && col0 + 2 * j + 1 < p.No) ? __ldg(p.bias + col0 + 2 * j + 1) : 0u;
+            bw[j] = lo | (hi << 16);
+          }
+        }
 #pragma unroll
         for (int j = 0; j < 32; ++j) {
           float x = __uint_as_float(r[j]);
-          if (p.bias != nullptr && col0 + j < p.No)
-            x = __fadd_rn(x, __half2float(__ushort_as_half(__ldg(p.bias + col0 + j))));
+          if (p.bias != nullptr) {
+            const uint16_t hb = (uint16_t)((j & 1) ? (bw[j >> 1] >> 16) : (bw[j >> 1] & 0xFFFFu));
+            x = __fadd_rn(x, __half2float(__ushort_as_half(hb)));
+          }
           if (p.act != 0) {
             x = x > 0.0f ? x : 0.0f;
             if (p.act == 2) x = x < p.clip ? x : p.clip;
@@ -137,18 +195,12 @@ __device__ __forceinline__ uint32_t epilogue_tile(const GemmParams& p, uint32_t 
         const __half2 v = __floats2half2_rn(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1]));
         h[j] = *reinterpret_cast<const uint32_t*>(&v);
       }
-      if (p.mask != nullptr && p.act != 0 && row_ok) {
+      if (pass_bits != nullptr) {
         // data-gradient flavour: keep the value only where the layer input passes the activation
-        const uint16_t* mrow = p.mask + (int64_t)row * p.ldmask + col0;
+        const uint32_t bits = pass_bits[c];
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          bool pass = false;
-          if (col0 + j < p.No) {
-            const float y = __half2float(__ushort_as_half(__ldg(mrow + j)));
-            pass = p.act == 2 ? (y > 0.0f && y < p.clip) : (y > 0.0f);
-          }
-          if (!pass) h[j >> 1] &= (j & 1) ? 0x0000FFFFu : 0xFFFF0000u;
-        }
+        for (int j = 0; j < 32; ++j)
+          if (!((bits >> j) & 1u)) h[j >> 1] &= (j & 1) ? 0x0000FFFFu : 0xFFFF0000u;
       }
       if (row_ok) {
         uint16_t* dst = p.out + (int64_t)row * p.ldo + col0;
@@ -316,10 +368,14 @@ mp_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       const int m0 = (tile / p.n_tiles) * BM, n0 = (tile % p.n_tiles) * BN;
       const int acc = iter & 1;
       const uint32_t acc_phase = (iter >> 1) & 1;
+      const int row = m0 + q * 32 + lane;
+      uint32_t pass_bits[BN / 32];
+      const bool masked = p.mask != nullptr && p.act != 0 && p.out_mode != OUT_PARTIAL;
+      if (masked) load_pass_bits(p, row, n0, pass_bits);      // runs under the tile's main loop
       if (!ptx::mbar_wait(&bars->tmem_full[acc], acc_phase)) { ok = false; break; }
       ptx::tc_fence_after_sync();
-      const int row = m0 + q * 32 + lane;
-      const uint32_t bad = epilogue_tile(p, tmem_base + acc * BN + ((uint32_t)(q * 32) << 16), row, n0, split);
+      const uint32_t bad = epilogue_tile(p, tmem_base + acc * BN + ((uint32_t)(q * 32) << 16), row, n0, split,
+                                         masked ? pass_bits : nullptr);
       if (p.out_mode == OUT_F16_FLAG && p.flag != nullptr) {
         if (__any_sync(0xFFFFFFFFu, bad != 0) && lane == 0) atomicOr(p.flag, 1);
       }
@@ -505,11 +561,15 @@ mp_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a,
       const int m0 = (tile / p.n_tiles) * 256 + 128 * (int)rank, n0 = (tile % p.n_tiles) * BN;
       const int acc = iter & 1;
       const uint32_t acc_phase = (iter >> 1) & 1;
+      const int row = m0 + q * 32 + lane;
+      uint32_t pass_bits[BN / 32];
+      const bool masked = p.mask != nullptr && p.act != 0 && p.out_mode != OUT_PARTIAL;
+      if (masked) load_pass_bits(p, row, n0, pass_bits);      // runs under the tile's main loop
       if (!ptx::mbar_wait(&bars->tmem_full[acc], acc_phase)) { ok = false; break; }
       ptx::tc_fence_after_sync();
-      const int row = m0 + q * 32 + lane;
       const uint32_t bad =
-          epilogue_tile(p, tmem_base + acc * BN + ((uint32_t)(q * 32) << 16), row, n0, split);
+          epilogue_tile(p, tmem_base + acc * BN + ((uint32_t)(q * 32) << 16), row, n0, split,
+                        masked ? pass_bits : nullptr);
       if (p.out_mode == OUT_F16_FLAG && p.flag != nullptr) {
         if (__any_sync(0xFFFFFFFFu, bad != 0) && lane == 0) atomicOr(p.flag, 1);
       }
