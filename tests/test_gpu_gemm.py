@@ -174,3 +174,31 @@ def test_argument_errors(mp):
     with pytest.raises(mp.MpError) as e:
         mp.mp_linear_bwd_wgrad(big, dy, dw, None, None)                   # workspace missing
     assert e.value.code == mp.MP_ERR_NOMEM
+
+
+def test_results_do_not_depend_on_timing(mp):
+    """Split reductions add their partial sums in a fixed order and nothing uses atomics on
+    values, so repeated launches on the same inputs give identical bits (a race in the pipeline
+    or in the split path would show up here as a difference)."""
+    g = torch.Generator(device="cuda"); g.manual_seed(3)
+    for (M, K, N) in [(3000, 200, 296), (8192, 1024, 1024), (4096, 128, 256)]:
+        X = (torch.randn(M, K, generator=g, device="cuda")).half()
+        dY = (torch.randn(M, N, generator=g, device="cuda") * 8).half()
+        W = (torch.randn(K, N, generator=g, device="cuda") / 16).half()
+        ws = torch.empty(max(max(mp.mp_gemm_workspace_bytes(M, K, N, o) for o in range(3)), 16),
+                         dtype=torch.uint8, device="cuda")
+        ref = None
+        for rep in range(4):
+            dW = torch.zeros(K, N, dtype=torch.float16, device="cuda")
+            dX = torch.zeros(M, K, dtype=torch.float16, device="cuda")
+            Y = torch.zeros(M, N, dtype=torch.float16, device="cuda")
+            ws.fill_(rep)                                   # stale scratch contents must not matter
+            mp.mp_linear_bwd_wgrad(X, dY, dW, None, ws)
+            mp.mp_linear_bwd_dgrad(dY, W, dX, ws)
+            mp.mp_linear_fwd(X, W, Y, ws)
+            out = [t.view(torch.int16).clone() for t in (dW, dX, Y)]
+            if ref is None:
+                ref = out
+            else:
+                assert all(torch.equal(a, b) for a, b in zip(ref, out))
+    assert mp.mp_gemm_device_status() == 0

@@ -363,3 +363,18 @@ def test_state_checkpoint_and_resume(orc, mp):
     assert torch.equal(Ta.w16.view(torch.int16), Tc.w16.view(torch.int16))
     for s_, p_ in ((sa, pa), (sb, pb), (sc2, pc)):
         s_.close(); p_.close()
+
+
+def test_log_ring_wraps(mp):
+    """More steps than the ring holds: the newest MP_LOG_CAPACITY records come back, oldest first."""
+    st = mp.State(init_scale=4.0, growth_interval=1000)
+    n = mp.MP_LOG_CAPACITY + 137
+    for _ in range(n):
+        mp.mp_loss_scale_update(st)
+    log = st.read_log()
+    assert len(log) == mp.MP_LOG_CAPACITY
+    assert [r.step for r in log] == list(range(n - mp.MP_LOG_CAPACITY, n))
+    assert st.read().step == n and st.read().t == n
+    few = st.read_log(5)
+    assert [r.step for r in few] == list(range(n - 5, n))
+    st.close()
