@@ -149,6 +149,7 @@ class LinearStack:
             self.step(xs, gs)
         self.events = saved
         self.graph = g
+        return g
 
     def replay(self):
         self.graph.replay()
@@ -227,3 +228,67 @@ class LinearStack:
     def close(self):
         self.plan.close()
         self.state.close()
+
+
+class HostPipeline:
+    """Host-fed steps with the copies of the next batch under the step of the current one.
+
+    Two sets of device staging buffers alternate.  submit() copies one batch from pinned host
+    memory into the idle set on a copy stream; run() waits for the oldest submitted batch, runs
+    the step on it (a CUDA graph per staging set, recorded the first time the set is used) and
+    returns the loss-scale state read back from the device.  With one batch submitted ahead,
+        submit(b0); for i: submit(b[i+1]); state = run()
+    the host-to-device copy of batch i+1 overlaps the kernels of batch i; every batch is still
+    copied and every state still read, only not one after the other.  No arithmetic here."""
+
+    def __init__(self, stack: LinearStack, use_graph: bool = True):
+        s = self.stack = stack
+        self.use_graph = use_graph
+        self.copy_stream = torch.cuda.Stream(device=s.device)
+        mk_x = lambda l: None if s.chained[l] else torch.zeros(
+            s.shapes[l][0], _align(s.shapes[l][1]), dtype=torch.float16, device=s.device)
+        mk_g = lambda l: None if s.feeds_next(l) else torch.zeros(
+            s.shapes[l][0], s.shapes[l][2], dtype=torch.float32, device=s.device)
+        self.x_in = [[mk_x(l) for l in range(s.L)] for _ in range(2)]
+        self.g_in = [[mk_g(l) for l in range(s.L)] for _ in range(2)]
+        self.ready = [None, None]        # event: the set's copies have landed
+        self.consumed = [None, None]     # event: the step that read the set has finished
+        self.graphs = [None, None]
+        self.fill, self.drain, self.pending = 0, 0, 0
+
+    def submit(self, xs_host, gs_host):
+        """Starts the copies of one batch (pinned host tensors, one per layer that takes input)."""
+        assert self.pending < 2, "both staging sets are in use: call run() first"
+        s, k = self.stack, self.fill
+        cs = self.copy_stream
+        if self.consumed[k] is not None:
+            cs.wait_event(self.consumed[k])          # the step that read this set must be over
+        with torch.cuda.stream(cs):
+            for l in range(s.L):
+                if self.x_in[k][l] is not None:
+                    self.x_in[k][l][:, :s.shapes[l][1]].copy_(xs_host[l], non_blocking=True)
+                if self.g_in[k][l] is not None:
+                    self.g_in[k][l].copy_(gs_host[l], non_blocking=True)
+            self.ready[k] = torch.cuda.Event()
+            self.ready[k].record(cs)
+        self.fill, self.pending = k ^ 1, self.pending + 1
+
+    def run(self):
+        """Runs the step on the oldest submitted batch and returns the device state after it."""
+        assert self.pending > 0, "nothing submitted"
+        s, k = self.stack, self.drain
+        main = torch.cuda.current_stream()
+        main.wait_event(self.ready[k])
+        if self.use_graph and self.graphs[k] is None:
+            s.step(self.x_in[k], self.g_in[k])       # this batch's step, call by call
+            saved = s.graph
+            self.graphs[k] = s.capture(self.x_in[k], self.g_in[k], warmup=0)   # recorded, not run
+            s.graph = saved
+        elif self.use_graph:
+            self.graphs[k].replay()
+        else:
+            s.step(self.x_in[k], self.g_in[k])
+        self.consumed[k] = torch.cuda.Event()
+        self.consumed[k].record(main)
+        self.drain, self.pending = k ^ 1, self.pending - 1
+        return s.state.read()

@@ -254,6 +254,50 @@ def test_graph_replay_equals_call_by_call(orc, mp):
     a.close(); b.close()
 
 
+def test_host_pipeline_equals_serial_host_steps(orc, mp):
+    """Batches fed from pinned host memory through the double-buffered pipeline (copy of batch
+    i+1 under the step of batch i, one CUDA graph per staging set) leave bit-for-bit the state
+    of the same batches copied and stepped one after the other, overflow batch included."""
+    from paper_1805_10387_b200.stack import LinearStack, HostPipeline
+    cfg = synth.config("c1")
+    L = len(cfg.shapes)
+    chained = [cfg.chained(l) for l in range(L)]
+
+    def make():
+        st = LinearStack(cfg.shapes, chained, lr=cfg.lr, init_scale=cfg.init_scale, growth_interval=3)
+        for l in range(L):
+            w = synth.weights(cfg, l)
+            st.load_weights(l, torch.from_numpy(w).cuda(),
+                            torch.from_numpy(synth.fp16_bits(w).view(np.float16).reshape(w.shape)).cuda())
+        return st
+    a, b = make(), make()
+    steps = 9
+    batches = []
+    for s in range(steps):
+        x = torch.from_numpy(synth.activations(cfg, 0, s).view(np.float16)).pin_memory()
+        g = synth.upstream(cfg, 1, s).copy()
+        if s == 4:
+            g[3, 5] = np.inf
+        batches.append(([x, None], [None, torch.from_numpy(g).pin_memory()]))
+    states_a = [a.step_from_host(xs, gs) for xs, gs in batches]          # serial, call by call
+    pipe = HostPipeline(b, use_graph=True)
+    states_b = []
+    pipe.submit(*batches[0])
+    for s in range(steps):
+        if s + 1 < steps:
+            pipe.submit(*batches[s + 1])
+        states_b.append(pipe.run())
+    key = lambda h: (h.scale, h.t, h.skipped, h.step, h.good_steps)
+    assert [key(h) for h in states_a] == [key(h) for h in states_b]
+    assert states_a[-1].skipped == 1 and states_a[-1].step == steps
+    for fa, fb in ((a.w32_flat, b.w32_flat), (a.m_flat, b.m_flat), (a.v_flat, b.v_flat)):
+        assert torch.equal(fa.view(torch.int32), fb.view(torch.int32))
+    assert torch.equal(a.w16_flat.view(torch.int16), b.w16_flat.view(torch.int16))
+    with pytest.raises(AssertionError):
+        pipe.run()                                   # nothing submitted
+    a.close(); b.close()
+
+
 @pytest.mark.parametrize("name,shapes,acts,clip", [
     ("c3", [(384, 136, 520), (384, 520, 136), (384, 136, 136)], [1, 0, 0], 20.0),       # ReLU inside the FFN pair
     ("c4", [(512, 200, 200)] * 3 + [(512, 200, 29)], [2, 2, 2, 0], 20.0),              # clipped ReLU chain
