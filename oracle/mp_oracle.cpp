@@ -368,6 +368,10 @@ void orc_momentum_update(const uint16_t* g16, float* w32, float* u, uint16_t* w1
 // iteration's inspection.  Halve on overflow, double after `interval` clean steps
 // in a row, clamp to [s_min, s_max].  dynamic == 0: S never changes (static loss
 // scaling), but the counters still advance.
+// Second policy, not in the paper (which only names "Backoff"): with tolerance H > 1 the
+// scale is halved at the H-th overflow since it last changed, so that an isolated overflow
+// costs one skipped step but no precision; every overflow step is still skipped and still
+// restarts the count of clean steps.  H = 1 is the plain policy.
 struct orc_scaler {
   float S;
   float s_min, s_max;
@@ -377,19 +381,26 @@ struct orc_scaler {
   int64_t t;          // applied optimizer steps
   int64_t step;       // all steps
   int64_t skipped;    // overflow steps
+  int32_t tolerance;  // overflows that it takes to halve S (1: every overflow halves)
+  int32_t strikes;    // overflows since S last changed
 };
 
 void orc_scaler_update(orc_scaler* s, int found_inf) {
   if (found_inf) {
     s->skipped += 1;
     s->good = 0;
-    if (s->dynamic) s->S = std::max(s->S * 0.5f, s->s_min);
+    s->strikes += 1;
+    if (s->dynamic && s->strikes >= s->tolerance) {
+      s->S = std::max(s->S * 0.5f, s->s_min);
+      s->strikes = 0;
+    }
   } else {
     s->t += 1;
     s->good += 1;
     if (s->dynamic && s->good >= s->interval) {
       s->S = std::min(s->S * 2.0f, s->s_max);
       s->good = 0;
+      s->strikes = 0;
     }
   }
   s->step += 1;

@@ -37,7 +37,8 @@ def build(force: bool = False) -> str:
 class _Scaler(C.Structure):
     _fields_ = [("S", C.c_float), ("s_min", C.c_float), ("s_max", C.c_float),
                 ("interval", C.c_int32), ("dynamic", C.c_int32), ("good", C.c_int32),
-                ("t", C.c_int64), ("step", C.c_int64), ("skipped", C.c_int64)]
+                ("t", C.c_int64), ("step", C.c_int64), ("skipped", C.c_int64),
+                ("tolerance", C.c_int32), ("strikes", C.c_int32)]
 
 
 _lib = None
@@ -253,11 +254,13 @@ def momentum_update(g16, w32, u, w16, S, lr, mu, weight_decay=0.0):
 
 
 class Scaler:
-    """Loss-scale state machine: halve on overflow, double after `interval` clean steps."""
+    """Loss-scale state machine: halve at the `tolerance`-th overflow since S last changed
+    (1: at every overflow), double after `interval` clean steps in a row."""
 
     def __init__(self, init_scale=65536.0, interval=1000, s_min=1.0, s_max=2.0 ** 24,
-                 dynamic=True):
-        self.c = _Scaler(init_scale, s_min, s_max, interval, 1 if dynamic else 0, 0, 0, 0, 0)
+                 dynamic=True, tolerance=1):
+        self.c = _Scaler(init_scale, s_min, s_max, interval, 1 if dynamic else 0, 0, 0, 0, 0,
+                         tolerance, 0)
 
     def update(self, flag: int):
         lib().orc_scaler_update(C.byref(self.c), int(flag))
@@ -267,6 +270,7 @@ class Scaler:
     t = property(lambda self: int(self.c.t))
     step = property(lambda self: int(self.c.step))
     skipped = property(lambda self: int(self.c.skipped))
+    strikes = property(lambda self: int(self.c.strikes))
 
 
 # ------------------------------------------------------------ step driver

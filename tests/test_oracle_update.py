@@ -188,3 +188,31 @@ def test_scaler_closed_form_from_flag_sequence(orc):
                 log2s, run = min(log2s + 1, 24), 0
         s.update(int(f))
         assert s.S == 2.0 ** log2s and s.good == run
+
+
+def test_scaler_overflow_tolerance_golden_and_invariants(orc):
+    """Second policy: halve at the H-th overflow since S last changed."""
+    rows = [tuple(int(x) for x in l.split()) for l in open(os.path.join(GOLD, "scaler_tolerance2_trajectory.txt"))
+            if l.strip() and not l.startswith("#")]
+    s = orc.Scaler(init_scale=2.0 ** 10, interval=3, tolerance=2)
+    for step, flag, log2s in rows:
+        s.update(flag)
+        assert s.S == 2.0 ** log2s, step
+    assert s.skipped == sum(f for _, f, _ in rows) and s.t == len(rows) - s.skipped
+    # n overflows in a row from a fresh state halve floor(n / H) times; every one is skipped
+    for H in (1, 2, 3, 5):
+        for n in range(0, 12):
+            s = orc.Scaler(init_scale=2.0 ** 20, interval=1000, tolerance=H)
+            for _ in range(n):
+                s.update(1)
+            assert s.S == 2.0 ** (20 - n // H) and s.skipped == n and s.t == 0 and s.strikes == n % H
+    # isolated overflows, each followed by a doubling, never halve when H >= 2
+    s = orc.Scaler(init_scale=2.0 ** 10, interval=2, tolerance=2)
+    for rep in range(5):
+        s.update(1); assert s.S == 2.0 ** (10 + rep)
+        s.update(0); s.update(0); assert s.S == 2.0 ** (11 + rep) and s.strikes == 0
+    # static mode: nothing moves S, counters still advance
+    s = orc.Scaler(init_scale=10.0, interval=2, dynamic=False, tolerance=2)
+    for f in (1, 1, 1, 0, 0):
+        s.update(f); assert s.S == 10.0
+    assert s.skipped == 3 and s.t == 2
