@@ -52,13 +52,18 @@ typedef struct mp_update_plan mp_update_plan; /* device table over the tensors o
 /* Loss-scale policy (Section 3.1, item 1).  dynamic != 0: halve S (not below min_scale) after
  * a step whose gradients held an inf/NaN, double it (not above max_scale) after
  * growth_interval clean steps in a row.  dynamic == 0: S stays init_scale (static loss
- * scaling); an overflow step is still skipped. */
+ * scaling); an overflow step is still skipped.
+ * overflow_tolerance = H > 1 selects a second policy that the paper does not describe: S is
+ * halved at the H-th overflow since S last changed (a doubling clears the count too), so an
+ * isolated overflow costs a skipped step but no halving.  Every overflow step is still
+ * skipped and still restarts the run of clean steps.  H = 1 is the plain rule. */
 typedef struct {
   float init_scale;        /* > 0 */
   float min_scale;         /* > 0 */
   float max_scale;         /* >= min_scale */
   int32_t growth_interval; /* >= 1 */
   int32_t dynamic;
+  int32_t overflow_tolerance; /* >= 1 */
 } mp_scaler_config;
 
 typedef enum { MP_OPT_ADAM = 0, MP_OPT_MOMENTUM = 1 } mp_opt_kind;
@@ -80,6 +85,8 @@ typedef struct {
   int32_t good_steps;  /* clean steps since S last changed                                  */
   int32_t found_inf;   /* flag accumulated by the current step so far                       */
   int32_t status;      /* MP_OK or the first device-side error (MP_ERR_TIMEOUT)             */
+  int32_t overflow_tolerance;
+  int32_t strikes;     /* overflows since S last changed (always 0 with tolerance 1)        */
   int64_t t;           /* applied optimizer steps                                           */
   int64_t step;        /* all steps                                                         */
   int64_t skipped;     /* overflow steps                                                    */

@@ -384,13 +384,18 @@ __global__ void mp_loss_scale_update_kernel(mp_dev_state* st) {
   if (h.found_inf != 0) {
     h.skipped += 1;
     h.good_steps = 0;
-    if (h.dynamic) h.scale = fmaxf(__fmul_rn(h.scale, 0.5f), h.min_scale);
+    h.strikes += 1;
+    if (h.dynamic && h.strikes >= h.overflow_tolerance) {
+      h.scale = fmaxf(__fmul_rn(h.scale, 0.5f), h.min_scale);
+      h.strikes = 0;
+    }
   } else {
     h.t += 1;
     h.good_steps += 1;
     if (h.dynamic && h.good_steps >= h.growth_interval) {
       h.scale = fminf(__fmul_rn(h.scale, 2.0f), h.max_scale);
       h.good_steps = 0;
+      h.strikes = 0;
     }
   }
   h.found_inf = 0;
@@ -438,7 +443,7 @@ int64_t mp_kernel_launch_count(void) { return mp::g_launches.load(); }
 int mp_state_create(const mp_scaler_config* cfg, mp_state** out) {
   if (!cfg || !out) return mp::set_error(MP_ERR_INVALID_ARG, "mp_state_create: null argument");
   if (!(cfg->init_scale > 0) || !(cfg->min_scale > 0) || !(cfg->max_scale >= cfg->min_scale) ||
-      cfg->growth_interval < 1)
+      cfg->growth_interval < 1 || cfg->overflow_tolerance < 1)
     return mp::set_error(MP_ERR_INVALID_ARG, "mp_state_create: bad scaler configuration");
   if (int rc = mp::check_device()) return rc;
   mp_state* s = new (std::nothrow) mp_state{nullptr, 0};
@@ -456,6 +461,7 @@ int mp_state_create(const mp_scaler_config* cfg, mp_state** out) {
   h.max_scale = cfg->max_scale;
   h.growth_interval = cfg->growth_interval;
   h.dynamic = cfg->dynamic ? 1 : 0;
+  h.overflow_tolerance = cfg->overflow_tolerance;
   cudaError_t e = cudaMemcpy(s->dev, &h, sizeof(h), cudaMemcpyHostToDevice);
   if (e != cudaSuccess) {
     cudaFree(s->dev);

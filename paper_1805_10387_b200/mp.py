@@ -31,7 +31,8 @@ class MpError(RuntimeError):
 
 class ScalerConfig(C.Structure):
     _fields_ = [("init_scale", C.c_float), ("min_scale", C.c_float), ("max_scale", C.c_float),
-                ("growth_interval", C.c_int32), ("dynamic", C.c_int32)]
+                ("growth_interval", C.c_int32), ("dynamic", C.c_int32),
+                ("overflow_tolerance", C.c_int32)]
 
 
 class OptimConfig(C.Structure):
@@ -42,7 +43,8 @@ class OptimConfig(C.Structure):
 class StateHost(C.Structure):
     _fields_ = [("scale", C.c_float), ("min_scale", C.c_float), ("max_scale", C.c_float),
                 ("growth_interval", C.c_int32), ("dynamic", C.c_int32), ("good_steps", C.c_int32),
-                ("found_inf", C.c_int32), ("status", C.c_int32), ("t", C.c_int64),
+                ("found_inf", C.c_int32), ("status", C.c_int32),
+                ("overflow_tolerance", C.c_int32), ("strikes", C.c_int32), ("t", C.c_int64),
                 ("step", C.c_int64), ("skipped", C.c_int64)]
 
 
@@ -275,8 +277,9 @@ class State:
     """Owner of an mp_state handle (device-resident loss-scale state)."""
 
     def __init__(self, init_scale=65536.0, growth_interval=1000, min_scale=1.0,
-                 max_scale=2.0 ** 24, dynamic=True):
-        cfg = ScalerConfig(init_scale, min_scale, max_scale, growth_interval, 1 if dynamic else 0)
+                 max_scale=2.0 ** 24, dynamic=True, overflow_tolerance=1):
+        cfg = ScalerConfig(init_scale, min_scale, max_scale, growth_interval, 1 if dynamic else 0,
+                           overflow_tolerance)
         h = C.c_void_p()
         _check(lib().mp_state_create(C.byref(cfg), C.byref(h)))
         self.handle = h

@@ -24,7 +24,7 @@ class LinearStack:
     def __init__(self, shapes, chained, optimizer="adam", lr=1e-3, beta1=0.9, beta2=0.999,
                  eps=1e-8, momentum=0.9, weight_decay=0.0, init_scale=65536.0,
                  growth_interval=1000, min_scale=1.0, max_scale=2.0 ** 24, dynamic=True,
-                 device="cuda", acts=None, clip=20.0, bias=False):
+                 device="cuda", acts=None, clip=20.0, bias=False, overflow_tolerance=1):
         """acts[l]: mp.MP_ACT_* after layer l's product (a layer whose output feeds no chained
         layer must have MP_ACT_NONE); bias: every layer gets a bias vector."""
         self.shapes = [tuple(s) for s in shapes]
@@ -38,7 +38,8 @@ class LinearStack:
         self.device = torch.device(device)
         self.opt = mp.OptimConfig(mp.MP_OPT_ADAM if optimizer == "adam" else mp.MP_OPT_MOMENTUM,
                                   lr, beta1, beta2, eps, momentum, weight_decay)
-        self.state = mp.State(init_scale, growth_interval, min_scale, max_scale, dynamic)
+        self.state = mp.State(init_scale, growth_interval, min_scale, max_scale, dynamic,
+                              overflow_tolerance)
 
         # parameters, moments and weight gradients live in flat buffers; every tensor starts on
         # a 16-byte boundary and rows are padded to a multiple of 8 elements

@@ -378,3 +378,30 @@ def test_log_ring_wraps(mp):
     few = st.read_log(5)
     assert [r.step for r in few] == list(range(n - 5, n))
     st.close()
+
+
+@pytest.mark.parametrize("H", [1, 2, 3])
+def test_scaler_overflow_tolerance(orc, mp, H):
+    """Second policy (halve at the H-th overflow since S last changed) against the oracle on a
+    seeded flag sequence with bursts, isolated overflows and doublings."""
+    rng = np.random.default_rng(40 + H)
+    flags = (rng.uniform(size=300) < 0.15).astype(int).tolist() + [1] * 7 + [0] * 9 + [1, 0, 0, 0, 1, 1]
+    st = mp.State(init_scale=2.0 ** 12, growth_interval=3, min_scale=2.0 ** 6, max_scale=2.0 ** 15,
+                  overflow_tolerance=H)
+    sc = orc.Scaler(2.0 ** 12, 3, 2.0 ** 6, 2.0 ** 15, tolerance=H)
+    one = torch.zeros(8, dtype=torch.float16, device="cuda")
+    bad = one.clone(); bad[5] = float("inf")
+    want = []
+    for f in flags:
+        mp.mp_check_finite(bad if f else one, st)
+        mp.mp_loss_scale_update(st)
+        sc.update(f)
+        want.append(sc.S)
+    log = st.read_log()
+    assert [r.scale_after for r in log] == want and [r.found_inf for r in log] == flags
+    h = st.read()
+    assert (h.scale, h.t, h.skipped, h.good_steps, h.strikes, h.overflow_tolerance) == \
+        (sc.S, sc.t, sc.skipped, sc.good, sc.strikes, H)
+    st.close()
+    with pytest.raises(Exception):
+        mp.State(overflow_tolerance=0)
