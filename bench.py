@@ -32,7 +32,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 
 # DRAM bytes per launch of the GEMM kernel from one ncu capture (dram__bytes_read.sum +
 # dram__bytes_write.sum), keyed by workload, valid only for the kernel source it was taken on.
-NCU_TRAFFIC = {"sha": "bfb5727f4250fe32", "bytes_per_launch": {"c2": 51.5e6}}
+NCU_TRAFFIC = {"sha": "91e17aeb87c979d5", "bytes_per_launch": {"c2": 77.0e6}}
 
 
 def peaks():

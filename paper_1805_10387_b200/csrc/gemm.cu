@@ -613,6 +613,10 @@ mp_splitk_reduce_kernel(const float* __restrict__ ws, int splits, int Mo, int No
   const int64_t total = (int64_t)Mo * vec_per_row;
   const int64_t split_stride = (int64_t)Mo * ws_ld;
   uint32_t bad = 0;
+  // Launched with programmatic stream serialization: the blocks may be resident before the
+  // product kernel has finished, and wait here until its partial sums are complete and visible.
+  ptx::launch_dependents();
+  ptx::grid_dependency_wait();
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total;
        i += (int64_t)gridDim.x * blockDim.x) {
     const int row = (int)(i / vec_per_row);
@@ -849,10 +853,18 @@ int run_gemm(const char* name, const Operand& A, const Operand& B, void* out, in
     const int64_t vecs = Mo * ((No + 3) / 4);
     int64_t blocks = (vecs + 255) / 256;
     if (blocks > (int64_t)sms * 8) blocks = (int64_t)sms * 8;
-    mp_splitk_reduce_kernel<<<(int)blocks, 256, 0, st>>>(p.ws, p.splits, p.Mo, p.No, p.ws_ld, p.out,
-                                                         p.ldo, want_flag ? flag : nullptr);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)blocks, 1, 1);
+    cfg.blockDim = dim3(256, 1, 1);
+    cfg.stream = st;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    MP_CUDA_TRY(cudaLaunchKernelEx(&cfg, mp_splitk_reduce_kernel, (const float*)p.ws, p.splits, p.Mo,
+                                   p.No, p.ws_ld, p.out, p.ldo, want_flag ? flag : (int*)nullptr));
     mp::count_launch();
-    MP_CUDA_TRY(cudaGetLastError());
   }
   return MP_OK;
 }
