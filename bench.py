@@ -456,6 +456,8 @@ def main():
                    "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": upd_gbs / pk["hbm_gbs"],
                    "frac_of_nominal_8000": upd_gbs / 8000.0, "bytes_per_param": bytes_per_param,
                    "avg_launch_ms": sum(applied_ms) / len(applied_ms), "peak_source": pk_src + " copy"},
+        # device time per call class per step in the call-by-call region (sum over the step's calls)
+        "breakdown_ms_per_step": {k: sum(v) / args.steps for k, v in sorted(per.items())},
         "clocks": clocks,
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
