@@ -318,55 +318,101 @@ mp_scale_upstream_kernel(const float* __restrict__ g32, uint16_t* __restrict__ o
   }
 }
 
-// Bias gradient, stage 1: FP32 column sums of dY over a slab of rows.  A block owns 64 columns
-// (one half2 per lane) and one slab; its 8 warps stride over the slab's rows, then add their
-// sums in warp order through shared memory.  partial[slab][n] is written once, no atomics.
-constexpr int kBiasSlabs = 64;
-__global__ void __launch_bounds__(kThreads)
+// Bias gradient, stage 1: FP32 column sums of dY over a slab of rows.  A block owns up to 256
+// columns and one slab.  A lane reads one 16-byte vector (8 columns) of a row; when a row has
+// fewer than 32 vectors the spare lanes of the warp take further rows (lane = row group *
+// vecs + vector), so narrow matrices still fill the warp.  The 8 warps stride over the slab's
+// rows, four rows in flight per thread; the per-thread sums are then added through shared
+// memory in (warp, row group) order.  partial[slab][n] is written once, no atomics, so the
+// result does not depend on timing.  Row pitches are multiples of 8, so a vector that starts
+// below N lies inside its row; columns at or beyond N are read and dropped.
+constexpr int kBiasSlabs = 512;
+constexpr int kBiasCols = 256;
+__global__ void __launch_bounds__(kThreads, 8)
 mp_bias_grad_partial_kernel(const uint16_t* __restrict__ dY, int64_t lddy, int64_t M, int64_t N,
-                            float* __restrict__ partial, int slabs) {
+                            float* __restrict__ partial, int slabs, int vecs) {
+  // vecs: vectors per row handled by one warp, a power of two <= 32
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int64_t col = (int64_t)blockIdx.x * 64 + lane * 2;
+  const int groups = 32 / vecs;                     // rows a warp reads at once
+  const int vc = lane & (vecs - 1), rg = lane / vecs;
+  const int64_t col = (int64_t)blockIdx.x * kBiasCols + vc * 8;
   const int slab = blockIdx.y;
   const int64_t rows_per = (M + slabs - 1) / slabs;
   const int64_t r0 = slab * rows_per, r1 = r0 + rows_per < M ? r0 + rows_per : M;
-  float a0 = 0.0f, a1 = 0.0f;
+  const int64_t stride = 8 * groups;                // rows between two reads of one thread
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // stage 2 may take its place early
+  float acc[8];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) acc[j] = 0.0f;
   if (col < N) {
-    const bool two = col + 1 < N;
-    for (int64_t r = r0 + warp; r < r1; r += 8) {
-      const uint16_t* src = dY + r * lddy + col;
-      if (two) {
-        const uint32_t w = *reinterpret_cast<const uint32_t*>(src);
-        a0 = __fadd_rn(a0, half_bits_to_float((uint16_t)(w & 0xFFFFu)));
-        a1 = __fadd_rn(a1, half_bits_to_float((uint16_t)(w >> 16)));
-      } else {
-        a0 = __fadd_rn(a0, half_bits_to_float(src[0]));
+    const uint16_t* base = dY + col;
+    for (int64_t r = r0 + warp * groups + rg; r < r1; r += 4 * stride) {
+      uint4 v[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int64_t rr = r + stride * u;
+        v[u] = rr < r1 ? __ldcs(reinterpret_cast<const uint4*>(base + rr * lddy)) : make_uint4(0, 0, 0, 0);
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {          // ascending rows; a row past the slab adds +0
+        const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          acc[2 * j] = __fadd_rn(acc[2 * j], half_bits_to_float((uint16_t)(w[j] & 0xFFFFu)));
+          acc[2 * j + 1] = __fadd_rn(acc[2 * j + 1], half_bits_to_float((uint16_t)(w[j] >> 16)));
+        }
       }
     }
   }
-  __shared__ float s0[8][32], s1[8][32];
-  s0[warp][lane] = a0;
-  s1[warp][lane] = a1;
-  __syncthreads();
-  if (warp == 0 && col < N) {
-    float t0 = s0[0][lane], t1 = s1[0][lane];
+  __shared__ float sm[8][8][32];             // [warp][element][lane]
 #pragma unroll
-    for (int w = 1; w < 8; ++w) { t0 = __fadd_rn(t0, s0[w][lane]); t1 = __fadd_rn(t1, s1[w][lane]); }
-    partial[(int64_t)slab * N + col] = t0;
-    if (col + 1 < N) partial[(int64_t)slab * N + col + 1] = t1;
+  for (int j = 0; j < 8; ++j) sm[warp][j][lane] = acc[j];
+  __syncthreads();
+  // thread (warp = element j, lane = vector) adds the sums of column col + j over the warps
+  // and their row groups in a fixed order
+  const int j = warp;
+  if (lane < vecs) {
+    float t = 0.0f;
+    for (int w = 0; w < 8; ++w)
+      for (int g = 0; g < groups; ++g) t = __fadd_rn(t, sm[w][j][g * vecs + lane]);
+    const int64_t c = (int64_t)blockIdx.x * kBiasCols + lane * 8 + j;
+    if (c < N) partial[(int64_t)slab * N + c] = t;
   }
 }
 
-// Bias gradient, stage 2: add the slabs in ascending order, round to FP16, store, inspect.
-__global__ void __launch_bounds__(kThreads)
+// Bias gradient, stage 2: add the slabs in a fixed order, round to FP16, store, inspect.  A block
+// of 1024 threads owns 32 columns; thread (group, column) adds its share of the slabs in
+// ascending order, eight loads in flight at a time, then the 32 groups are added in ascending
+// order through shared memory.
+constexpr int kBiasFinalThreads = 1024;
+__global__ void __launch_bounds__(kBiasFinalThreads)
 mp_bias_grad_final_kernel(const float* __restrict__ partial, int slabs, int64_t N,
                           uint16_t* __restrict__ db, mp_dev_state* st) {
-  const int64_t n = (int64_t)blockIdx.x * kThreads + threadIdx.x;
-  uint32_t bad = 0;
+  const int lane = threadIdx.x & 31, grp = threadIdx.x >> 5;
+  const int64_t n = (int64_t)blockIdx.x * 32 + lane;
+  const int per = (slabs + 31) / 32;
+  asm volatile("griddepcontrol.wait;" ::: "memory");   // stage 1 complete, its sums visible
+  const int s_begin = grp * per;
+  const int s_end = s_begin + per < slabs ? s_begin + per : slabs;
+  float a = 0.0f;
   if (n < N) {
-    float a = partial[n];
-    for (int s = 1; s < slabs; ++s) a = __fadd_rn(a, partial[(int64_t)s * N + n]);
-    const uint16_t h = float_to_half_bits(a);
+    for (int s0 = s_begin; s0 < s_end; s0 += 8) {
+      float v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) v[u] = s0 + u < s_end ? partial[(int64_t)(s0 + u) * N + n] : 0.0f;
+#pragma unroll
+      for (int u = 0; u < 8; ++u) a = __fadd_rn(a, v[u]);
+    }
+  }
+  __shared__ float sm[32][32];
+  sm[grp][lane] = a;
+  __syncthreads();
+  uint32_t bad = 0;
+  if (grp == 0 && n < N) {
+    float t = sm[0][lane];
+#pragma unroll
+    for (int g = 1; g < 32; ++g) t = __fadd_rn(t, sm[g][lane]);
+    const uint16_t h = float_to_half_bits(t);
     db[n] = h;
     bad = ((h & 0x7C00u) == 0x7C00u) ? 1u : 0u;
   }
@@ -638,14 +684,28 @@ int mp_scale_upstream(const float* g32, void* dY16, int64_t n, const mp_state* s
   return MP_OK;
 }
 
-static int bias_slabs(int64_t M) {
-  const int64_t want = (M + 255) / 256;
+// Slabs of rows that the first stage sums separately: at most eight blocks per SM (the kernel is
+// compiled to fit eight), all resident at
+// once (a grid a little larger than what fits runs a second, nearly empty round), each with at
+// least 32 rows (8 warps x 4 rows in flight), at most kBiasSlabs.
+static int bias_vecs(int64_t N) {        // 16-byte vectors per row and warp, as a power of two
+  int vecs = 1;
+  while (vecs < 32 && (int64_t)vecs * 8 < N) vecs *= 2;
+  return vecs;
+}
+
+static int bias_slabs(int64_t M, int64_t N) {
+  const int64_t col_blocks = (N + kBiasCols - 1) / kBiasCols;
+  int64_t want = 8 * 148 / col_blocks;
+  const int64_t rows_per_pass = 32 * (32 / bias_vecs(N));     // rows one block reads at once
+  const int64_t by_rows = (M + rows_per_pass - 1) / rows_per_pass;
+  if (want > by_rows) want = by_rows;
   return (int)(want < 1 ? 1 : (want > kBiasSlabs ? kBiasSlabs : want));
 }
 
 size_t mp_bias_grad_workspace_bytes(int64_t M, int64_t N) {
   if (M <= 0 || N <= 0) return 0;
-  return (size_t)bias_slabs(M) * (size_t)N * sizeof(float);
+  return (size_t)bias_slabs(M, N) * (size_t)N * sizeof(float);
 }
 
 int mp_bias_grad(const void* dY16, int64_t lddy, void* db16, int64_t M, int64_t N, mp_state* state,
@@ -658,15 +718,24 @@ int mp_bias_grad(const void* dY16, int64_t lddy, void* db16, int64_t M, int64_t 
   if (!workspace || workspace_bytes < need)
     return mp::set_error(MP_ERR_NOMEM, "mp_bias_grad: workspace of %zu bytes needed", need);
   if (int rc = mp::check_device()) return rc;
-  const int slabs = bias_slabs(M);
+  const int slabs = bias_slabs(M, N);
   cudaStream_t st = (cudaStream_t)stream;
-  const dim3 grid((unsigned)((N + 63) / 64), (unsigned)slabs);
+  const dim3 grid((unsigned)((N + kBiasCols - 1) / kBiasCols), (unsigned)slabs);
+  const int vecs = bias_vecs(N);
   mp_bias_grad_partial_kernel<<<grid, kThreads, 0, st>>>((const uint16_t*)dY16, lddy, M, N,
-                                                        (float*)workspace, slabs);
-  mp_bias_grad_final_kernel<<<(unsigned)((N + kThreads - 1) / kThreads), kThreads, 0, st>>>(
-      (const float*)workspace, slabs, N, (uint16_t*)db16, state ? state->dev : nullptr);
+                                                        (float*)workspace, slabs, vecs);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)((N + 31) / 32), 1, 1);
+  cfg.blockDim = dim3(kBiasFinalThreads, 1, 1);
+  cfg.stream = st;
+  cudaLaunchAttribute attr;            // resident early, waits on the device for stage 1
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  MP_CUDA_TRY(cudaLaunchKernelEx(&cfg, mp_bias_grad_final_kernel,
+      (const float*)workspace, slabs, N, (uint16_t*)db16, state ? state->dev : (mp_dev_state*)nullptr));
   mp::count_launch(2);
-  MP_CUDA_TRY(cudaGetLastError());
   return MP_OK;
 }
 
