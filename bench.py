@@ -2,6 +2,7 @@
 """Benchmark of the mixed-precision training step of a linear-layer stack on B200.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2|c3|c4|c5] [--impl reference]
+  python bench.py --workload c3 --per-shape      (each layer shape's products alone, beside cuBLAS)
 
 One step = forward, weight-gradient and data-gradient products of every layer (FP16 operands,
 FP32 accumulation), upstream scaling, the fused unscale / inspect / FP32-master optimizer /
@@ -9,7 +10,8 @@ FP16 recast update and the loss-scale state machine, on one batch of seeded synt
 Prints ONE JSON line.  `value` is the whole job's GEMM throughput over the step time (inputs
 resident in HBM); `e2e` is the same with pinned host inputs copied in and the loss-scale state
 read back every step; `roofline` is for the dominant kernel (the tcgen05 GEMM), timed with CUDA
-events around each launch inside the timed region; `update` gives the fused update's GB/s.
+events around a region that replays the step's product calls alone; `update` gives the fused
+update's GB/s.
 `--impl reference` times the CPU oracle (the slow, plain restatement of the method) instead.
 """
 from __future__ import annotations
@@ -32,7 +34,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 
 # DRAM bytes per launch of the GEMM kernel from one ncu capture (dram__bytes_read.sum +
 # dram__bytes_write.sum), keyed by workload, valid only for the kernel source it was taken on.
-NCU_TRAFFIC = {"sha": "91e17aeb87c979d5", "bytes_per_launch": {"c2": 77.0e6}}
+NCU_TRAFFIC = {"sha": "53b5ce8b8635f328", "bytes_per_launch": {"c2": 74.6e6}}
 
 
 def peaks():
@@ -241,6 +243,71 @@ def run_update_sweep(args):
         "sweep": rows, "clocks": clocks}))
 
 
+# ------------------------------------------------------------------ per-shape timing
+def run_per_shape(args):
+    """Each distinct layer shape of the workload alone: the three products back to back inside a
+    CUDA graph of 24 launches over rotating operand sets (working set above the 126 MB L2), best
+    of five replays, with torch.matmul (cuBLAS) on the same operands beside it as a reference
+    point.  Prints one JSON line; not the bench value (no power-capped steady state)."""
+    import torch
+    from paper_1805_10387_b200 import mp, synth
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    mp.lib()
+    cfg = synth.config(args.workload)
+    reps = 24
+
+    def graph_us(fn, sets):
+        side = torch.cuda.Stream()
+        with torch.cuda.stream(side):
+            for i in range(3):
+                fn(i % sets)
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=side):
+                for i in range(reps):
+                    fn(i % sets)
+            g.replay()
+            torch.cuda.synchronize()
+            best = float("inf")
+            for _ in range(5):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                g.replay()
+                b.record()
+                torch.cuda.synchronize()
+                best = min(best, a.elapsed_time(b) / reps)
+        return best * 1e3
+
+    rows = []
+    for (M, K, N) in sorted(set(cfg.shapes), key=cfg.shapes.index):
+        Np = (N + 7) // 8 * 8
+        sets = max(2, int(300e6 // (2 * (M * K + K * Np + M * Np))) + 1)
+        mk = lambda r, c, scale: [(torch.randn(r, c, device="cuda") * scale).half() for _ in range(sets)]
+        X, W, dY = mk(M, K, 1.0), mk(K, Np, K ** -0.5), mk(M, Np, 0.01)
+        out = lambda r, c: [torch.empty(r, c, device="cuda", dtype=torch.float16) for _ in range(sets)]
+        Y, dX, dW = out(M, Np), out(M, K), out(K, Np)
+        ws = torch.empty(max(16, max(mp.mp_gemm_workspace_bytes(M, K, N, op) for op in (0, 1, 2))),
+                         dtype=torch.uint8, device="cuda")
+        st = mp.State()
+        us = {"fwd": graph_us(lambda i: mp.mp_linear_fwd(X[i], W[i][:, :N], Y[i][:, :N], ws), sets),
+              "dgrad": graph_us(lambda i: mp.mp_linear_bwd_dgrad(dY[i][:, :N], W[i][:, :N], dX[i], ws), sets),
+              "wgrad": graph_us(lambda i: mp.mp_linear_bwd_wgrad(X[i], dY[i][:, :N], dW[i][:, :N], st, ws), sets)}
+        if N == Np:
+            us["cublas_fwd"] = graph_us(lambda i: torch.matmul(X[i], W[i], out=Y[i]), sets)
+            us["cublas_dgrad"] = graph_us(lambda i: torch.matmul(dY[i], W[i].t(), out=dX[i]), sets)
+            us["cublas_wgrad"] = graph_us(lambda i: torch.matmul(X[i].t(), dY[i], out=dW[i]), sets)
+        rows.append({"M": M, "K": K, "N": N, "operand_sets": sets,
+                     "us": {k: round(v, 1) for k, v in us.items()},
+                     "tflops": {k: round(2.0 * M * K * N / v / 1e6) for k, v in us.items()}})
+        st.close()
+        del X, W, dY, Y, dX, dW, ws
+        torch.cuda.empty_cache()
+    assert mp.mp_gemm_device_status() == 0
+    print(json.dumps({"per_shape": rows, "workload": cfg.name, "launches_per_graph": reps}))
+
+
 # ------------------------------------------------------------------ CUDA arm
 def main():
     ap = argparse.ArgumentParser()
@@ -252,12 +319,16 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--real-layers", action="store_true",
                     help="biases on every layer and an activation inside every chain (ReLU; clipped ReLU for c4)")
+    ap.add_argument("--per-shape", action="store_true",
+                    help="time each distinct layer shape's three products alone, beside torch.matmul")
     ap.add_argument("--max-params", type=float, default=1e9, help="c5: largest parameter count of the sweep")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
     if args.workload == "c5":
         return run_update_sweep(args)
+    if args.per_shape:
+        return run_per_shape(args)
 
     import numpy as np
     import torch
@@ -363,14 +434,51 @@ def main():
     ms_total = timed(run_step, args.steps)
     st1 = stack.state.read()
     launches = launches_per_step * args.steps
-    # (B) the same steps launched call by call with a CUDA-event pair around every launch:
-    # per-kernel times for the roofline (the event records cost ~6 % of the step, so this
-    # region is not the one `value` is taken from)
-    stack.events = []
-    st0b = stack.state.read()
-    ms_events = timed(lambda: stack.step(xs, gs), args.steps)
-    events, stack.events = stack.events, None
-    st1b = stack.state.read()
+    # (B) per-call device times for the roofline.  One GPU: the same step recorded once more with
+    # an event-record node before and after every call; each timed replay is followed at once by
+    # an untimed one, so the device never idles while the host reads the events (a timed replay
+    # runs in the same power and clock state as the steps of (A); the event nodes themselves
+    # stop a kernel's prologue from overlapping its predecessor's tail, so this region is a
+    # little slower than (A) and is not the one `value` is taken from).  Several GPUs: call by
+    # call with an event pair around every launch.
+    per = {}
+    gemm_only = None
+    if use_graph:
+        # the products alone: the step's forward, weight-gradient and data-gradient calls (same
+        # order, same buffers) recorded without the other calls and without event nodes, replayed
+        # back to back: elapsed device time / launches = the GEMM kernels' average launch
+        # duration with their prologue overlap intact and no event between them
+        gemm_only = {}
+        for key, classes in (("gemm", ("fwd", "dgrad", "wgrad")), ("fwd", ("fwd",)), ("dgrad", ("dgrad",)),
+                             ("wgrad", ("wgrad",))):
+            n0 = mp.mp_kernel_launch_count()
+            g_sub = stack.capture_only(xs, gs, classes)
+            n_launch = mp.mp_kernel_launch_count() - n0
+            for _ in range(3):
+                g_sub.replay()
+            gemm_only[key] = (timed(g_sub.replay, args.steps) / args.steps, n_launch)
+        g_timed, ev = stack.capture_timed(xs, gs)
+        done = torch.cuda.Event()
+
+        def timed_steps():
+            for _ in range(args.steps):
+                g_timed.replay()
+                done.record()
+                stack.replay()
+                done.synchronize()
+                for name, a, b in ev:
+                    per.setdefault(name, []).append(a.elapsed_time(b))
+        ms_events = timed(timed_steps, 1) / 2.0
+        timed_how = ("a second timed region: the step's graph recorded with an event-record node before and "
+                     "after every call, each timed replay followed by an untimed one")
+    else:
+        stack.events = []
+        ms_events = timed(lambda: stack.step(xs, gs), args.steps)
+        events, stack.events = stack.events, None
+        for name, a, b in events:
+            per.setdefault(name, []).append(a.elapsed_time(b))
+        timed_how = ("a second timed region of the same steps, launched call by call with a CUDA-event "
+                     "pair around every launch")
     # (C) end to end: pinned host inputs in, loss-scale state out, every step
     # through the double-buffered host pipeline: the copies of batch i+1 run under the kernels of
     # batch i; every step still copies its inputs in and reads the state back
@@ -399,26 +507,33 @@ def main():
     clocks = sampler.stop() if rank == 0 else None
     assert mp.mp_gemm_device_status() == 0, "a GEMM kernel reported a device-side error"
 
-    # per-call device times from the events recorded inside the timed region
-    per = {}
-    for name, a, b in events:
-        per.setdefault(name, []).append(a.elapsed_time(b))
     flops_step = cfg.gemm_flops()
     ms_step = ms_total / args.steps
     value = world * flops_step / (ms_step * 1e-3) / 1e12
     e2e_val = world * flops_step / (ms_e2e / args.steps * 1e-3) / 1e12
     pk, pk_src = peaks()
-    gemm_ms = sum(sum(per.get(k, [])) for k in ("fwd", "dgrad", "wgrad"))
     gemm_calls = sum(len(per.get(k, [])) for k in ("fwd", "dgrad", "wgrad"))
+    if gemm_only is not None:
+        gemm_ms = gemm_only["gemm"][0] * args.steps
+        gemm_launches = gemm_only["gemm"][1] * args.steps
+        per_op = {k: (flops_step / 3) / (gemm_only[k][0] * 1e-3) / 1e12 for k in ("fwd", "dgrad", "wgrad")}
+        gemm_how = ("the step's product calls alone (same order and buffers, no other call, no event between "
+                    "them) as a CUDA graph replayed back to back for the same number of steps; CUDA events "
+                    "around the region; launches include the split-reduction kernels of the weight gradients")
+    else:
+        gemm_ms = sum(sum(per.get(k, [])) for k in ("fwd", "dgrad", "wgrad"))
+        gemm_launches = gemm_calls
+        per_op = {k: (flops_step / 3) * args.steps / (sum(per[k]) * 1e-3) / 1e12
+                  for k in ("fwd", "dgrad", "wgrad") if k in per}
+        gemm_how = timed_how
     gemm_tflops = flops_step * args.steps / (gemm_ms * 1e-3) / 1e12
     skipped = st1.skipped - st0.skipped
-    skipped_b = st1b.skipped - st0b.skipped
     bytes_per_param = 28 if cfg.optimizer == "adam" else 20
     upd_ms = per.get("update", [0.0])
-    applied = [t for t in upd_ms]
     upd_bytes = cfg.n_params() * bytes_per_param
-    # skipped steps return at once; GB/s is quoted on the applied ones only
-    applied_ms = sorted(applied)[skipped_b:] if skipped_b < len(applied) else applied
+    # a skipped step's update returns at once (a few microseconds); GB/s is quoted on the
+    # applied ones only
+    applied_ms = [t for t in upd_ms if t >= 0.25 * max(upd_ms)]
     upd_gbs = upd_bytes / (sum(applied_ms) / len(applied_ms) * 1e-3) / 1e9
     sha = kernel_sha()
     traffic = NCU_TRAFFIC["bytes_per_launch"].get(args.workload) if NCU_TRAFFIC["sha"] == sha else None
@@ -438,7 +553,7 @@ def main():
         "gpu_launches": int(launches),
         "launch_mode": "one CUDA graph replay per step (captured from the same C-ABI calls)" if use_graph
                        else "call by call",
-        "ms_per_step_call_by_call_with_events": ms_events / args.steps,
+        "ms_per_step_in_event_timed_region": ms_events / args.steps,
         "skipped_steps_in_timed_region": int(skipped),
         "loss_scale": st1.scale,
         "roofline": {"kernel": "mp_gemm_pair_kernel", "bound": "tensor", "achieved": gemm_tflops,
@@ -447,16 +562,16 @@ def main():
                      "peak_source": f"{pk_src} cuBLAS bf16 sustained (fp16 nominal ratio 1.0)",
                      "frac_of_burst_peak": gemm_tflops / pk["bf16_tflops"],
                      "frac_of_nominal_2250": gemm_tflops / 2250.0,
-                     "launches": gemm_calls, "avg_launch_ms": gemm_ms / max(gemm_calls, 1),
-                     "timed_in": "a second timed region of the same steps, launched call by call with a "
-                                 "CUDA-event pair around every launch",
-                     "per_op_tflops": {k: (flops_step / 3) * args.steps / (sum(per[k]) * 1e-3) / 1e12
-                                       for k in ("fwd", "dgrad", "wgrad") if k in per}},
+                     "launches": gemm_launches, "avg_launch_ms": gemm_ms / max(gemm_launches, 1),
+                     "calls": gemm_calls, "timed_in": gemm_how,
+                     "per_op_tflops": per_op},
         "update": {"kernel": "mp_master_update_kernel", "bound": "hbm", "achieved": upd_gbs,
                    "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": upd_gbs / pk["hbm_gbs"],
                    "frac_of_nominal_8000": upd_gbs / 8000.0, "bytes_per_param": bytes_per_param,
                    "avg_launch_ms": sum(applied_ms) / len(applied_ms), "peak_source": pk_src + " copy"},
-        # device time per call class per step in the call-by-call region (sum over the step's calls)
+        # device time per call class per step from the event-timed region (sum over the step's
+        # calls; every call's interval is stretched by its two event nodes, a few microseconds)
+        "breakdown_timed_in": timed_how,
         "breakdown_ms_per_step": {k: sum(v) / args.steps for k, v in sorted(per.items())},
         "clocks": clocks,
     }

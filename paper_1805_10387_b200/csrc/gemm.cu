@@ -94,6 +94,18 @@ __device__ __forceinline__ void report_timeout(B* bars) {
   atomicCAS(&g_gemm_status, 0, (int)MP_ERR_TIMEOUT);
 }
 
+// Width of the MMAs of the tile whose first column is n_base: the columns that exist, rounded up
+// to 32, at most BN.  A ragged last column tile (1600 = 6 x 256 + 64) then issues a quarter of
+// the MMA work of a full one instead of multiplying zero-filled columns, and the producer
+// fetches only the B boxes those MMAs read (a full tile's loads, 64 B per clock and SM, take
+// as long as its MMAs, so a narrow tile gets faster only if its loads shrink too).  Multiples
+// of 32 keep every form legal: N % 16 == 0 for both instruction shapes, and each CTA of a pair
+// holds N / 2 (a multiple of 16) columns of B.
+__device__ __forceinline__ int tile_width(int No, int n_base) {
+  const int left = No - n_base;
+  return left >= BN ? BN : ((left + 31) & ~31);
+}
+
 // Epilogue of one 128 x 256 accumulator for one warp: this thread owns output row `row`
 // (TMEM lane) and walks the columns in chunks of 32.  tmem_acc is the TMEM address of the
 // accumulator's first column in this warp's lane quarter.  Returns nonzero if an inf or NaN
@@ -286,6 +298,7 @@ mp_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     for (int w = blockIdx.x; w < total_work && ok; w += gridDim.x) {
       const int split = w % p.splits, tile = w / p.splits;
       const int m0 = (tile / p.n_tiles) * BM, n0 = (tile % p.n_tiles) * BN;
+      const int b_boxes = B_MN ? (tile_width(p.No, n0) + 63) / 64 : BN / 64;   // 64-column boxes of B
       const int kb0 = (int)((int64_t)split * p.num_kb / p.splits);
       const int kb1 = (int)((int64_t)(split + 1) * p.num_kb / p.splits);
       for (int kb = kb0; kb < kb1; ++kb) {
@@ -293,7 +306,7 @@ mp_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         if (lane == 0) {
           uint8_t* sA = smem + stage * STAGE_BYTES;
           uint8_t* sB = sA + A_BYTES;
-          ptx::mbar_arrive_expect_tx(&bars->full[stage], STAGE_BYTES);
+          ptx::mbar_arrive_expect_tx(&bars->full[stage], A_BYTES + b_boxes * CHUNK_BYTES);
           const int k = kb * BK;
           if (A_MN) {
 #pragma unroll
@@ -305,7 +318,8 @@ mp_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           if (B_MN) {
 #pragma unroll
             for (int c = 0; c < BN / 64; ++c)
-              ptx::tma_load_2d(sB + c * CHUNK_BYTES, &map_b, &bars->full[stage], n0 + 64 * c, k);
+              if (c < b_boxes)
+                ptx::tma_load_2d(sB + c * CHUNK_BYTES, &map_b, &bars->full[stage], n0 + 64 * c, k);
           } else {
             ptx::tma_load_2d(sB, &map_b, &bars->full[stage], k, n0);
           }
@@ -327,13 +341,14 @@ mp_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer
-    constexpr uint32_t idesc = ptx::idesc_f16_f32(BM, BN, A_MN, B_MN);
     int stage = 0;
     uint32_t phase = 0;
     int iter = 0;
     bool ok = true;
     for (int w = blockIdx.x; w < total_work && ok; w += gridDim.x, ++iter) {
-      const int split = w % p.splits;
+      const int split = w % p.splits, tile = w / p.splits;
+      const uint32_t idesc =
+          ptx::idesc_f16_f32(BM, tile_width(p.No, (tile % p.n_tiles) * BN), A_MN, B_MN);
       const int kb0 = (int)((int64_t)split * p.num_kb / p.splits);
       const int kb1 = (int)((int64_t)(split + 1) * p.num_kb / p.splits);
       const int acc = iter & 1;
@@ -430,7 +445,8 @@ struct Barriers2 {
 template <bool A_MN, bool B_MN>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1)
 mp_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a,
-                    const __grid_constant__ CUtensorMap map_b, const GemmParams p) {
+                    const __grid_constant__ CUtensorMap map_b,
+                    const __grid_constant__ CUtensorMap map_b32, const GemmParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                              ~static_cast<uintptr_t>(1023));
@@ -453,6 +469,7 @@ mp_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a,
     ptx::fence_mbar_init();
     ptx::prefetch_tensormap(&map_a);
     ptx::prefetch_tensormap(&map_b);
+    if (!B_MN) ptx::prefetch_tensormap(&map_b32);
   }
   if (warp == 1) {
     ptx::tmem_alloc_pair(&bars->tmem_base, TMEM_COLS);
@@ -478,7 +495,15 @@ mp_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a,
     for (int w = pair; w < total_work && ok; w += npairs) {
       const int split = w % p.splits, tile = w / p.splits;
       const int m0 = (tile / p.n_tiles) * 256 + 128 * (int)rank;
-      const int n0 = (tile % p.n_tiles) * BN + 128 * (int)rank;
+      // this CTA's half of the tile's columns: 128 of a full tile, fewer of a narrow last one.
+      // B arrives in boxes of 64 columns (output dimension contiguous) or, for a narrow tile
+      // of a reduction-contiguous B, in boxes of 32 rows from the second tensor map; only the
+      // boxes that the MMAs read are fetched.
+      const int n_base = (tile % p.n_tiles) * BN;
+      const int half = tile_width(p.No, n_base) >> 1;
+      const int n0 = n_base + half * (int)rank;
+      const int b_boxes = B_MN ? (half + 63) / 64 : (half + 31) / 32;
+      const uint32_t b_bytes = B_MN ? b_boxes * CHUNK_BYTES : b_boxes * (32 * BK * 2);
       const int kb0 = (int)((int64_t)split * p.num_kb / p.splits);
       const int kb1 = (int)((int64_t)(split + 1) * p.num_kb / p.splits);
       for (int kb = kb0; kb < kb1; ++kb) {
@@ -491,7 +516,7 @@ mp_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a,
           // barrier before this arrive (the count of bytes still to come just goes negative
           // for a moment); they cannot reach it before the previous phase has completed,
           // because the peer refills a stage only after the MMAs that read it are done.
-          if (leader) ptx::mbar_arrive_expect_tx(&bars->full[stage], 2 * STAGE2_BYTES);
+          if (leader) ptx::mbar_arrive_expect_tx(&bars->full[stage], 2 * (HALF_BYTES + b_bytes));
           const int k = kb * BK;
           if (A_MN) {
             ptx::tma_load_2d_pair(sA, &map_a, full, m0, k);
@@ -501,9 +526,12 @@ mp_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a,
           }
           if (B_MN) {
             ptx::tma_load_2d_pair(sB, &map_b, full, n0, k);
-            ptx::tma_load_2d_pair(sB + CHUNK_BYTES, &map_b, full, n0 + 64, k);
-          } else {
+            if (b_boxes > 1) ptx::tma_load_2d_pair(sB + CHUNK_BYTES, &map_b, full, n0 + 64, k);
+          } else if (b_boxes == 4) {
             ptx::tma_load_2d_pair(sB, &map_b, full, k, n0);
+          } else {
+            for (int c = 0; c < b_boxes; ++c)   // 32 rows of 128 B each: 4 KiB apart, whole swizzle groups
+              ptx::tma_load_2d_pair(sB + c * (32 * BK * 2), &map_b32, full, k, n0 + 32 * c);
           }
         }
         __syncwarp();
@@ -525,13 +553,14 @@ mp_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a,
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer (leader CTA only)
     if (leader) {
-      constexpr uint32_t idesc = ptx::idesc_f16_f32(256, BN, A_MN, B_MN);
       int stage = 0;
       uint32_t phase = 0;
       int iter = 0;
       bool ok = true;
       for (int w = pair; w < total_work && ok; w += npairs, ++iter) {
-        const int split = w % p.splits;
+        const int split = w % p.splits, tile = w / p.splits;
+        const uint32_t idesc =
+            ptx::idesc_f16_f32(256, tile_width(p.No, (tile % p.n_tiles) * BN), A_MN, B_MN);
         const int kb0 = (int)((int64_t)split * p.num_kb / p.splits);
         const int kb1 = (int)((int64_t)(split + 1) * p.num_kb / p.splits);
         const int acc = iter & 1;
@@ -746,8 +775,8 @@ int launch(const CUtensorMap& ma, const CUtensorMap& mb, const GemmParams& p, in
 }
 
 template <bool A_MN, bool B_MN>
-int launch_pair(const CUtensorMap& ma, const CUtensorMap& mb, const GemmParams& p, int64_t work,
-                cudaStream_t st) {
+int launch_pair(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mb32,
+                const GemmParams& p, int64_t work, cudaStream_t st) {
   static int max_pairs = 0;
   if (max_pairs == 0) {
     MP_CUDA_TRY(cudaFuncSetAttribute(mp_gemm_pair_kernel<A_MN, B_MN>,
@@ -777,7 +806,7 @@ int launch_pair(const CUtensorMap& ma, const CUtensorMap& mb, const GemmParams& 
   attr.val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = &attr;
   cfg.numAttrs = 1;
-  MP_CUDA_TRY(cudaLaunchKernelEx(&cfg, mp_gemm_pair_kernel<A_MN, B_MN>, ma, mb, p));
+  MP_CUDA_TRY(cudaLaunchKernelEx(&cfg, mp_gemm_pair_kernel<A_MN, B_MN>, ma, mb, mb32, p));
   mp::count_launch();
   return MP_OK;
 }
@@ -823,11 +852,17 @@ int run_gemm(const char* name, const Operand& A, const Operand& B, void* out, in
                            workspace ? ws_bytes : (size_t)0);
   }
 
-  CUtensorMap ma, mb;
+  CUtensorMap ma, mb, mb32;
   if (int rc = A.mn_major ? make_map(&ma, A.ptr, A.mn, A.red, A.ld, 64, BK)
                           : make_map(&ma, A.ptr, A.red, A.mn, A.ld, BK, BM)) return rc;
   if (int rc = B.mn_major ? make_map(&mb, B.ptr, B.mn, B.red, B.ld, 64, BK)
                           : make_map(&mb, B.ptr, B.red, B.mn, B.ld, BK, pair ? 128 : BN)) return rc;
+  // reduction-contiguous B of the pair kernel: 32-row boxes for a narrow last column tile
+  if (pair && !B.mn_major) {
+    if (int rc = make_map(&mb32, B.ptr, B.red, B.mn, B.ld, BK, 32)) return rc;
+  } else {
+    mb32 = mb;
+  }
 
   int dev = 0, sms = 0;
   MP_CUDA_TRY(cudaGetDevice(&dev));
@@ -837,10 +872,10 @@ int run_gemm(const char* name, const Operand& A, const Operand& B, void* out, in
 
   int rc;
   if (pair) {
-    if (A.mn_major && B.mn_major) rc = launch_pair<true, true>(ma, mb, p, work, st);
-    else if (!A.mn_major && B.mn_major) rc = launch_pair<false, true>(ma, mb, p, work, st);
-    else if (!A.mn_major && !B.mn_major) rc = launch_pair<false, false>(ma, mb, p, work, st);
-    else rc = launch_pair<true, false>(ma, mb, p, work, st);
+    if (A.mn_major && B.mn_major) rc = launch_pair<true, true>(ma, mb, mb32, p, work, st);
+    else if (!A.mn_major && B.mn_major) rc = launch_pair<false, true>(ma, mb, mb32, p, work, st);
+    else if (!A.mn_major && !B.mn_major) rc = launch_pair<false, false>(ma, mb, mb32, p, work, st);
+    else rc = launch_pair<true, false>(ma, mb, mb32, p, work, st);
   } else {
     if (A.mn_major && B.mn_major) rc = launch<true, true>(ma, mb, p, grid, st);
     else if (!A.mn_major && B.mn_major) rc = launch<false, true>(ma, mb, p, grid, st);

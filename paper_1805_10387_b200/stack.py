@@ -119,15 +119,23 @@ class LinearStack:
     events = None   # set to a list to collect (name, start_event, end_event)
     grad_sync = None  # data-parallel runs: callable that all-reduces the flat FP16 gradient
 
+    only = None       # set to a set of call classes to make step() issue only those calls
+
     def _call(self, name, fn, *args):
+        if self.only is not None and name not in self.only:
+            return
         if self.events is None:
             fn(*args)
             return
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ext = self._events_external
+        a = torch.cuda.Event(enable_timing=True, external=ext)
+        b = torch.cuda.Event(enable_timing=True, external=ext)
         a.record()
         fn(*args)
         b.record()
         self.events.append((name, a, b))
+
+    _events_external = False
 
     # ---- CUDA graph of the step (removes the per-call host cost of ~40 launches per step) ----
     graph = None
@@ -154,6 +162,42 @@ class LinearStack:
 
     def replay(self):
         self.graph.replay()
+
+    def capture_only(self, xs, gs, classes):
+        """Records into a CUDA graph only the step's calls of the given classes ("fwd", "dgrad",
+        "wgrad", "scale", "update", "scaler"), in the step's order and on the step's buffers.
+        Replaying it back to back and dividing the elapsed device time by the number of
+        launches gives the average duration of those kernels without any event node or host
+        gap between them.  Call capture() first."""
+        assert self.graph is not None, "capture() first"
+        saved_events, saved_only = self.events, self.only
+        self.events, self.only = None, set(classes)
+        g = torch.cuda.CUDAGraph()
+        try:
+            with torch.cuda.graph(g):
+                self.step(xs, gs)
+        finally:
+            self.events, self.only = saved_events, saved_only
+        return g
+
+    def capture_timed(self, xs, gs):
+        """Records the step once more with an event-record node before and after every C-ABI
+        call and returns (graph, [(call class, start event, end event)]).  After a replay has
+        finished, start.elapsed_time(end) is the device time of that call inside the replayed
+        step: no host launch gaps, unlike events around call-by-call launches.  Every replay
+        overwrites the events, so read them before the next one.  Call capture() first (it
+        runs the library's one-time set-up outside any capture)."""
+        assert self.graph is not None, "capture() first"
+        saved = self.events
+        self.events, self._events_external = [], True
+        g = torch.cuda.CUDAGraph()
+        try:
+            with torch.cuda.graph(g):
+                self.step(xs, gs)
+            ev = self.events
+        finally:
+            self.events, self._events_external = saved, False
+        return g, ev
 
     def step_from_host(self, xs_host, gs_host):
         """The step as a caller with host data makes it: pinned host inputs are copied to the
@@ -204,7 +248,8 @@ class LinearStack:
                 n = self.shapes[l][2]
                 if self.dy[l].shape[1] == n:
                     self._call("scale", mp.mp_scale_upstream, gs[l], self.dy[l], self.state)
-                else:   # padded rows: scale into a dense buffer, then place (copy only)
+                elif self.only is None or "scale" in self.only:
+                    # padded rows: scale into a dense buffer, then place (copy only)
                     tmp = torch.empty(self.shapes[l][0], n, dtype=torch.float16, device=self.device)
                     mp.mp_scale_upstream(gs[l], tmp, self.state)
                     self.dy[l][:, :n].copy_(tmp)
@@ -220,7 +265,7 @@ class LinearStack:
             else:       # the layer below is activated: mask with its stored output (= this layer's input)
                 self._call("dgrad", mp.mp_linear_bwd_dgrad_act, self.dY(l), self.W16(l), X, self.dX(l),
                            below, self.clip, self.workspace)
-        if self.grad_sync is not None:       # data parallel: sum the FP16 gradients over ranks,
+        if self.grad_sync is not None and self.only is None:   # data parallel: sum the FP16 gradients over ranks,
             self.grad_sync(self.dw_flat)     # then inspect the reduced gradients in the update call
         self._call("update", mp.mp_master_update, self.plan, self.state, self.opt,
                    0 if self.grad_sync is None else 1)

@@ -96,6 +96,22 @@ def test_integer_exact_bitwise(orc, mp, op, M, K, N):
     assert bad.size == 0, (bad[:5], got[tuple(bad[0])], want[tuple(bad[0])])
 
 
+@pytest.mark.parametrize("op", ["fwd", "dgrad", "wgrad"])
+@pytest.mark.parametrize("width", [8, 40, 72, 96, 136, 168, 200, 232, 256 + 24, 256 + 104])
+def test_every_width_of_the_last_column_tile(orc, mp, op, width):
+    """The last column tile is multiplied only as wide as it is (rounded up to 32 columns):
+    every such width, for each operand layout, on the CTA-pair kernel (more than 128 output
+    rows) and on the one-CTA kernel."""
+    rng = np.random.default_rng(width)
+    for rows in (300, 70):
+        M, K, N = {"fwd": (rows, 136, width), "dgrad": (rows, width, 136), "wgrad": (136, rows, width)}[op]
+        sa, sb = _shapes_for(op, M, K, N)
+        A, B = _h(rng.integers(-2, 3, sa)), _h(rng.integers(-2, 3, sb))
+        got, _ = _run(mp, op, A, B)
+        want = _oracle(orc, op, A, B)
+        assert got.shape == want.shape and (got == want).all(), (op, rows, width)
+
+
 @pytest.mark.parametrize("op,M,K,N", [("wgrad", 4096, 128, 256), ("wgrad", 3000, 200, 300),
                                       ("fwd", 2048, 2048, 512), ("dgrad", 1500, 640, 2048)])
 def test_integer_exact_large_and_split(orc, mp, op, M, K, N):
