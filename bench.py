@@ -34,7 +34,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 
 # DRAM bytes per launch of the GEMM kernel from one ncu capture (dram__bytes_read.sum +
 # dram__bytes_write.sum), keyed by workload, valid only for the kernel source it was taken on.
-NCU_TRAFFIC = {"sha": "53b5ce8b8635f328", "bytes_per_launch": {"c2": 74.6e6}}
+NCU_TRAFFIC = {"sha": "c79dcfdfe0b8ac28", "bytes_per_launch": {"c2": 81.5e6}}
 
 
 def peaks():

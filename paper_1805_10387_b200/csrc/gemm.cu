@@ -5,9 +5,10 @@
 //   warp 1      MMA issuer: tcgen05.mma (FP16 x FP16 -> FP32) into tensor memory; owns the TMEM
 //               allocation (two 256-column accumulators, so the epilogue of one tile overlaps
 //               the main loop of the next)
-//   warps 2-5 (2-9 for the fused epilogues: two warps per TMEM lane quarter)   epilogue: tcgen05.ld, optional bias / activation / mask, round to FP16 (nearest
-//               even, overflow to inf), store; for the weight gradient also the inf/NaN
-//               inspection of what is stored
+//   warps 2-5   epilogue (warps 2-9 in the fused flavours, two per TMEM lane quarter): tcgen05.ld,
+//               optional bias / activation / mask, round to FP16 (nearest even, overflow to
+//               inf), stage in shared memory, TMA store; for the weight gradient also the
+//               inf/NaN inspection of what is stored
 //
 //   mp_gemm_pair_kernel  clusters of two CTAs, tcgen05.mma.cta_group::2, one 256 x 256 tile per
 //                        pair, 6 stages x 32 KiB per CTA; used for outputs of more than 128 rows
@@ -46,9 +47,9 @@ constexpr int CHUNK_BYTES = 64 * BK * 2;       // one 64 x 64 box of an MN-major
 // 137 against 154 us on the masked 25600x1600x1600 data gradient.
 constexpr int THREADS_PLAIN = 64 + 32 * 4;
 constexpr int THREADS_FUSED = 64 + 32 * 8;
-constexpr int THREADS = THREADS_FUSED;         // upper bound for __launch_bounds__
 constexpr int TMEM_COLS = 512;
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int STAGING_BYTES = 8 * 32 * 64 * 2;  // epilogue staging: 8 slots of 32 rows x 64 FP16 columns
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + STAGING_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 constexpr int kModelSMs = 148;                 // used by the split heuristic only
 
 __device__ int g_gemm_status = 0;              // first device-side error (bounded wait expired)
@@ -57,6 +58,7 @@ enum OutMode { OUT_F16 = 0, OUT_F16_FLAG = 1, OUT_PARTIAL = 2 };
 
 struct GemmParams {
   int Mo, No, R;        // output rows, output columns, reduction length
+  int No8;              // No rounded down to a multiple of 8: the columns the output tensor map covers
   int m_tiles, n_tiles, splits, num_kb;
   int out_mode;
   uint16_t* out;        // FP16 output [Mo, No], leading dimension ldo
@@ -106,10 +108,6 @@ __device__ __forceinline__ int tile_width(int No, int n_base) {
   return left >= BN ? BN : ((left + 31) & ~31);
 }
 
-// Epilogue of one 128 x 256 accumulator for one warp: this thread owns output row `row`
-// (TMEM lane) and walks the columns in chunks of 32.  tmem_acc is the TMEM address of the
-// accumulator's first column in this warp's lane quarter.  Returns nonzero if an inf or NaN
-// was stored as FP16.
 // Activation mask of one thread's row of a tile, one bit per column (word c = columns
 // 32c .. 32c+31): 1 where the layer input (the activated FP16 output of the layer below)
 // lies strictly inside the activation's linear range.  Called BEFORE the thread waits for the
@@ -152,19 +150,157 @@ __device__ __forceinline__ void load_pass_bits(const GemmParams& p, int row, int
   }
 }
 
-__device__ __forceinline__ uint32_t epilogue_tile(const GemmParams& p, uint32_t tmem_acc, int row,
-                                                  int n0, int split, int c_begin, int c_count,
+//
+// FP16 output leaves through shared memory: the warp's 32 rows x 64 columns (two chunks) are
+// written into a 4 KiB staging slot in the 128-byte-swizzled order of the output tensor map and
+// one TMA store moves the slot to global memory, whole 128-byte row segments at a time and
+// clipped at the matrix edges.  `stage` is this warp's slot area (nslots slots of 4 KiB,
+// 1024-byte aligned), `stores` its running count of committed stores, which picks the slot;
+// before a slot is rewritten the store that last read it must have finished reading.  A TMA
+// store clips the contiguous dimension in units of 16 bytes, not of elements, so the tensor map
+// covers only the first No8 = No rounded down to 8 columns; the up to 7 columns after them are
+// stored from registers.
+//
+// One warp per scheduler runs this, so its speed is set by the length of its dependent
+// instruction chains: the two chunks of a group are converted side by side, and the inf/NaN
+// test (weight gradient only) is two integer operations per packed pair.
+constexpr int SLOT_BYTES = 32 * 64 * 2;
+
+// One chunk (32 columns from col0) of this thread's row, FP16 modes: optional bias and
+// activation on the FP32 sums, rounding, optional activation mask, columns and rows that do not
+// exist, the inf/NaN test, the register-stored tail columns, and the 64 bytes of the row into
+// the staging slot (half = 0 / 1: first or second chunk of the 64-column group).
+template <bool FUSED>
+__device__ __forceinline__ void finish_chunk(const GemmParams& p, uint32_t (&r)[32], int col0, int row,
+                                             bool row_ok, int lane, uint8_t* slot, int half,
+                                             const uint32_t* pass_bits, int c, uint32_t& flag_acc) {
+  if (FUSED && (p.bias != nullptr || (p.act != 0 && p.mask == nullptr))) {
+    // forward flavour, on the FP32 values: + bias, then the activation
+    uint32_t bw[16];                          // 32 bias values as packed halves (0 if absent)
+    if (p.bias != nullptr && col0 + 32 <= p.No) {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {           // same address in every thread: one broadcast load
+        const uint4 q4 = __ldg(reinterpret_cast<const uint4*>(p.bias + col0) + j);
+        bw[4 * j] = q4.x; bw[4 * j + 1] = q4.y; bw[4 * j + 2] = q4.z; bw[4 * j + 3] = q4.w;
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < 16; ++j) {
+        const uint32_t lo = (p.bias != nullptr && col0 + 2 * j < p.No) ? __ldg(p.bias + col0 + 2 * j) : 0u;
+        const uint32_t hi = (p.bias != nullptr && col0 + 2 * j + 1 < p.No) ? __ldg(p.bias + col0 + 2 * j + 1) : 0u;
+        bw[j] = lo | (hi << 16);
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+      float x = __uint_as_float(r[j]);
+      if (p.bias != nullptr) {
+        const uint16_t hb = (uint16_t)((j & 1) ? (bw[j >> 1] >> 16) : (bw[j >> 1] & 0xFFFFu));
+        x = __fadd_rn(x, __half2float(__ushort_as_half(hb)));
+      }
+      if (p.act != 0) {
+        x = x > 0.0f ? x : 0.0f;
+        if (p.act == 2) x = x < p.clip ? x : p.clip;
+      }
+      r[j] = __float_as_uint(x);
+    }
+  }
+  uint32_t h[16];
+#pragma unroll
+  for (int j = 0; j < 16; ++j) {
+    const __half2 v = __floats2half2_rn(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1]));
+    h[j] = *reinterpret_cast<const uint32_t*>(&v);
+  }
+  if (FUSED && pass_bits != nullptr) {
+    // data-gradient flavour: keep the value only where the layer input passes the activation
+    const uint32_t bits = pass_bits[c];
+#pragma unroll
+    for (int j = 0; j < 32; ++j)
+      if (!((bits >> j) & 1u)) h[j >> 1] &= (j & 1) ? 0x0000FFFFu : 0xFFFF0000u;
+  }
+  if (col0 + 32 > p.No) {
+    // columns beyond No (dropped by the store) must not raise the flag: 0 x inf is NaN
+#pragma unroll
+    for (int j = 0; j < 32; ++j)
+      if (col0 + j >= p.No) h[j >> 1] &= (j & 1) ? 0x0000FFFFu : 0xFFFF0000u;
+  }
+  if (row_ok) {                               // rows beyond Mo are dropped by the store
+    if (p.out_mode == OUT_F16_FLAG) {
+      // a half is inf or NaN iff its exponent field is 0x7C00; adding 0x0400 to the isolated
+      // field then carries into bit 15 (and no further), for both halves of the word at once
+#pragma unroll
+      for (int j = 0; j < 16; ++j) flag_acc |= (h[j] & 0x7C007C00u) + 0x04000400u;
+    }
+    if (col0 + 32 > p.No8) {                  // the columns past the tensor map's last 16-byte unit
+      uint16_t* dst = p.out + (int64_t)row * p.ldo + col0;
+#pragma unroll
+      for (int j = 0; j < 32; ++j)
+        if (col0 + j >= p.No8 && col0 + j < p.No)
+          dst[j] = (uint16_t)((j & 1) ? (h[j >> 1] >> 16) : (h[j >> 1] & 0xFFFFu));
+    }
+  }
+  uint8_t* rowp = slot + lane * 128;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const int piece = half * 4 + j;           // 16-byte piece of the 128-byte row segment
+    *reinterpret_cast<uint4*>(rowp + ((piece ^ (lane & 7)) << 4)) =
+        make_uint4(h[4 * j], h[4 * j + 1], h[4 * j + 2], h[4 * j + 3]);
+  }
+}
+
+// Epilogue of one accumulator for one warp: this thread owns output row `row` (TMEM lane) and
+// the warp walks chunks c_begin .. c_begin + c_count (32 columns each, both even) of the tile
+// whose first column is n0.  tmem_acc is the TMEM address of the accumulator's first column in
+// this warp's lane quarter.  Returns nonzero if an inf or NaN was stored by the weight gradient.
+// The store half of a group: wait for the slot, round and stage both chunks, hand the slot over.
+template <bool FUSED>
+__device__ __forceinline__ void finish_group(const GemmParams& p, const CUtensorMap* map_out, uint8_t* stage,
+                                             int nslots, int& stores, uint32_t (&ra)[32], uint32_t (&rb)[32],
+                                             bool second, int colg, int g, int row, bool row_ok, int lane,
+                                             const uint32_t* pass_bits, uint32_t& flag_acc) {
+  uint8_t* slot = stage + (stores % nslots) * SLOT_BYTES;
+  // the slot must no longer be read by an earlier store
+  if (lane == 0) {
+    if (nslots == 2) ptx::bulk_wait_group_read<1>(); else ptx::bulk_wait_group_read<0>();
+  }
+  __syncwarp();
+  finish_chunk<FUSED>(p, ra, colg, row, row_ok, lane, slot, 0, pass_bits, 2 * g, flag_acc);
+  if (second) finish_chunk<FUSED>(p, rb, colg + 32, row, row_ok, lane, slot, 1, pass_bits, 2 * g + 1, flag_acc);
+  ptx::fence_proxy_async_smem();                // the slot is complete: hand it to the TMA unit
+  __syncwarp();
+  if (colg < p.No8) {                           // else: only register-stored columns in this group
+    if (lane == 0) {
+      ptx::tma_store_2d(map_out, slot, colg, row - lane);
+      ptx::bulk_commit_group();
+    }
+    ++stores;
+  }
+}
+
+// Epilogue of one accumulator for one warp: this thread owns output row `row` (TMEM lane) and
+// the warp walks chunks c_begin .. c_begin + c_count (32 columns each, both even) of the tile
+// whose first column is n0.  tmem_acc is the TMEM address of the accumulator's first column in
+// this warp's lane quarter.  Returns nonzero if an inf or NaN was stored by the weight gradient.
+// FUSED is the kernel's flavour (bias / activation / mask code present, eight epilogue warps);
+// the plain flavour carries none of that code: one warp per scheduler runs this, and a short
+// instruction stream matters more to it than anything else.
+template <bool FUSED>
+__device__ __forceinline__ uint32_t epilogue_tile(const GemmParams& p, const CUtensorMap* map_out,
+                                                  uint8_t* stage, int nslots, int& stores,
+                                                  uint32_t tmem_acc, int row, int n0, int split,
+                                                  int c_begin, int c_count,
                                                   const uint32_t* pass_bits = nullptr) {
   const bool row_ok = row < p.Mo;
-  uint32_t bad = 0;
+  const int lane = threadIdx.x & 31;
+  if (p.out_mode == OUT_PARTIAL) {
+    // FP32 partial sums of a split reduction: 128 contiguous bytes per thread and chunk
 #pragma unroll 1
-  for (int c = c_begin; c < c_begin + c_count; ++c) {
-    const int col0 = n0 + c * 32;
-    if (col0 >= p.No) break;                    // warp-uniform
-    uint32_t r[32];
-    ptx::tmem_ld_32x32(tmem_acc + c * 32, r);
-    ptx::tmem_ld_wait();
-    if (p.out_mode == OUT_PARTIAL) {
+    for (int c = c_begin; c < c_begin + c_count; ++c) {
+      const int col0 = n0 + c * 32;
+      if (col0 >= p.No) break;                  // warp-uniform
+      uint32_t r[32];
+      ptx::tmem_ld_32x32(tmem_acc + c * 32, r);
+      ptx::tmem_ld_wait();
       if (row_ok) {
         float* dst = p.ws + ((int64_t)split * p.Mo + row) * p.ws_ld + col0;
         if (col0 + 32 <= p.No) {
@@ -178,86 +314,39 @@ __device__ __forceinline__ uint32_t epilogue_tile(const GemmParams& p, uint32_t 
             if (col0 + j < p.No) dst[j] = __uint_as_float(r[j]);
         }
       }
-    } else {
-      const bool full_chunk = col0 + 32 <= p.No;
-      if (p.bias != nullptr || (p.act != 0 && p.mask == nullptr)) {
-        // forward flavour, on the FP32 values: + bias, then the activation
-        uint32_t bw[16];                          // 32 bias values as packed halves (0 if absent)
-        if (p.bias != nullptr && full_chunk) {
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {           // same address in every thread: one broadcast load
-            const uint4 q4 = __ldg(reinterpret_cast<const uint4*>(p.bias + col0) + j);
-            bw[4 * j] = q4.x; bw[4 * j + 1] = q4.y; bw[4 * j + 2] = q4.z; bw[4 * j + 3] = q4.w;
-          }
-        } else {
-#pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            const uint32_t lo = (p.bias != nullptr && col0 + 2 * j < p.No) ? __ldg(p.bias + col0 + 2 * j) : 0u;
-            const uint32_t hi = (p.bias != nullptr && col0 + 2 * j + 1 < p.No) ? __ldg(p.bias + col0 + 2 * j + 1) : 0u;
-            bw[j] = lo | (hi << 16);
-          }
-        }
-#pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          float x = __uint_as_float(r[j]);
-          if (p.bias != nullptr) {
-            const uint16_t hb = (uint16_t)((j & 1) ? (bw[j >> 1] >> 16) : (bw[j >> 1] & 0xFFFFu));
-            x = __fadd_rn(x, __half2float(__ushort_as_half(hb)));
-          }
-          if (p.act != 0) {
-            x = x > 0.0f ? x : 0.0f;
-            if (p.act == 2) x = x < p.clip ? x : p.clip;
-          }
-          r[j] = __float_as_uint(x);
-        }
-      }
-      uint32_t h[16];
-#pragma unroll
-      for (int j = 0; j < 16; ++j) {
-        const __half2 v = __floats2half2_rn(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1]));
-        h[j] = *reinterpret_cast<const uint32_t*>(&v);
-      }
-      if (pass_bits != nullptr) {
-        // data-gradient flavour: keep the value only where the layer input passes the activation
-        const uint32_t bits = pass_bits[c];
-#pragma unroll
-        for (int j = 0; j < 32; ++j)
-          if (!((bits >> j) & 1u)) h[j >> 1] &= (j & 1) ? 0x0000FFFFu : 0xFFFF0000u;
-      }
-      if (row_ok) {
-        uint16_t* dst = p.out + (int64_t)row * p.ldo + col0;
-        if (col0 + 32 <= p.No) {
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            *reinterpret_cast<uint4*>(dst + 8 * j) =
-                make_uint4(h[4 * j], h[4 * j + 1], h[4 * j + 2], h[4 * j + 3]);
-            bad |= pair_nonfinite(h[4 * j]) | pair_nonfinite(h[4 * j + 1]) |
-                   pair_nonfinite(h[4 * j + 2]) | pair_nonfinite(h[4 * j + 3]);
-          }
-        } else {
-#pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            if (col0 + j < p.No) {
-              const uint16_t hv = (uint16_t)((j & 1) ? (h[j >> 1] >> 16) : (h[j >> 1] & 0xFFFFu));
-              dst[j] = hv;
-              bad |= ((hv & 0x7C00u) == 0x7C00u) ? 1u : 0u;
-            }
-          }
-        }
-      }
     }
+    return 0;
   }
-  return bad;
+  if (row - lane >= p.Mo) return 0;             // nothing of this warp's rows exists
+  uint32_t flag_acc = 0;
+  // groups of 64 columns g_begin .. g_end that have columns (warp-uniform)
+  const int g_begin = c_begin >> 1;
+  int g_end = (c_begin + c_count) >> 1;
+  if (n0 + g_end * 64 > p.No) g_end = (p.No - n0 + 63) >> 6;
+  if (g_end <= g_begin) return 0;
+#pragma unroll 1
+  for (int g = g_begin; g < g_end; ++g) {
+    const int colg = n0 + g * 64;               // first column of the 64-column group
+    const bool second = colg + 32 < p.No;       // the group's second chunk has columns
+    uint32_t ra[32], rb[32];
+    ptx::tmem_ld_32x32(tmem_acc + g * 64, ra);
+    if (second) ptx::tmem_ld_32x32(tmem_acc + g * 64 + 32, rb);
+    ptx::tmem_ld_wait();
+    finish_group<FUSED>(p, map_out, stage, nslots, stores, ra, rb, second, colg, g, row, row_ok, lane,
+                        pass_bits, flag_acc);
+  }
+  return flag_acc & 0x80008000u;
 }
 
-template <bool A_MN, bool B_MN>
-__global__ void __launch_bounds__(THREADS, 1)
+template <bool A_MN, bool B_MN, bool WIDE>
+__global__ void __launch_bounds__(WIDE ? THREADS_FUSED : THREADS_PLAIN, 1)
 mp_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-               const GemmParams p) {
+               const __grid_constant__ CUtensorMap map_out, const GemmParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                              ~static_cast<uintptr_t>(1023));
-  Barriers* bars = reinterpret_cast<Barriers*>(smem + STAGES * STAGE_BYTES);
+  uint8_t* staging = smem + STAGES * STAGE_BYTES;
+  Barriers* bars = reinterpret_cast<Barriers*>(staging + STAGING_BYTES);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   ptx::launch_dependents();    // the next kernel's CTAs may take SMs as soon as ours leave them
 
@@ -274,6 +363,7 @@ mp_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     ptx::fence_mbar_init();
     ptx::prefetch_tensormap(&map_a);
     ptx::prefetch_tensormap(&map_b);
+    ptx::prefetch_tensormap(&map_out);
   }
   if (warp == 1) {
     ptx::tmem_alloc(&bars->tmem_base, TMEM_COLS);
@@ -388,6 +478,9 @@ mp_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const int q = warp & 3;                         // TMEM lane quarter this warp may read
     const int c_count = (BN / 32) / ((int)(blockDim.x / 32 - 2) / 4);   // column chunks per warp: 8 or 4
     const int c_begin = ((warp - 2) >> 2) * c_count;                    // its share of the tile's columns
+    const int nslots = 8 / ((int)blockDim.x / 32 - 2);                  // staging slots per warp: 2 or 1
+    uint8_t* stage = staging + (warp - 2) * nslots * SLOT_BYTES;
+    int stores = 0;
     int iter = 0;
     bool ok = true;
     for (int w = blockIdx.x; w < total_work && ok; w += gridDim.x, ++iter) {
@@ -401,7 +494,8 @@ mp_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       if (masked) load_pass_bits(p, row, n0, c_begin, c_count, pass_bits);   // runs under the tile's main loop
       if (!ptx::mbar_wait(&bars->tmem_full[acc], acc_phase)) { ok = false; break; }
       ptx::tc_fence_after_sync();
-      const uint32_t bad = epilogue_tile(p, tmem_base + acc * BN + ((uint32_t)(q * 32) << 16), row, n0, split,
+      const uint32_t bad = epilogue_tile<WIDE>(p, &map_out, stage, nslots, stores,
+                                         tmem_base + acc * BN + ((uint32_t)(q * 32) << 16), row, n0, split,
                                          c_begin, c_count, masked ? pass_bits : nullptr);
       if (p.out_mode == OUT_F16_FLAG && p.flag != nullptr) {
         if (__any_sync(0xFFFFFFFFu, bad != 0) && lane == 0) atomicOr(p.flag, 1);
@@ -410,6 +504,7 @@ mp_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       ptx::mbar_arrive(&bars->tmem_empty[acc]);
     }
     if (!ok) report_timeout(bars);
+    if (lane == 0) ptx::bulk_wait_group_all();   // this warp's output stores have left shared memory
   }
 
   // ---------------------------------------------------------------- teardown
@@ -431,7 +526,7 @@ mp_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 constexpr int STAGES2 = 6;
 constexpr int HALF_BYTES = 128 * BK * 2;            // 16 KiB: half a tile of A or of B
 constexpr int STAGE2_BYTES = 2 * HALF_BYTES;
-constexpr int SMEM2_BYTES = STAGES2 * STAGE2_BYTES + 1024 + 256;
+constexpr int SMEM2_BYTES = STAGES2 * STAGE2_BYTES + STAGING_BYTES + 1024 + 256;
 
 struct Barriers2 {
   uint64_t full[STAGES2];     // used in the leader: both CTAs' loads of a stage have landed
@@ -442,15 +537,17 @@ struct Barriers2 {
   volatile uint32_t abort;
 };
 
-template <bool A_MN, bool B_MN>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1)
+template <bool A_MN, bool B_MN, bool WIDE>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(WIDE ? THREADS_FUSED : THREADS_PLAIN, 1)
 mp_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a,
                     const __grid_constant__ CUtensorMap map_b,
-                    const __grid_constant__ CUtensorMap map_b32, const GemmParams p) {
+                    const __grid_constant__ CUtensorMap map_b32,
+                    const __grid_constant__ CUtensorMap map_out, const GemmParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                              ~static_cast<uintptr_t>(1023));
-  Barriers2* bars = reinterpret_cast<Barriers2*>(smem + STAGES2 * STAGE2_BYTES);
+  uint8_t* staging = smem + STAGES2 * STAGE2_BYTES;
+  Barriers2* bars = reinterpret_cast<Barriers2*>(staging + STAGING_BYTES);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = ptx::cluster_ctarank();
   const bool leader = rank == 0;
@@ -470,6 +567,7 @@ mp_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a,
     ptx::prefetch_tensormap(&map_a);
     ptx::prefetch_tensormap(&map_b);
     if (!B_MN) ptx::prefetch_tensormap(&map_b32);
+    ptx::prefetch_tensormap(&map_out);
   }
   if (warp == 1) {
     ptx::tmem_alloc_pair(&bars->tmem_base, TMEM_COLS);
@@ -597,6 +695,9 @@ mp_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a,
     const int q = warp & 3;
     const int c_count = (BN / 32) / ((int)(blockDim.x / 32 - 2) / 4);
     const int c_begin = ((warp - 2) >> 2) * c_count;
+    const int nslots = 8 / ((int)blockDim.x / 32 - 2);
+    uint8_t* stage = staging + (warp - 2) * nslots * SLOT_BYTES;
+    int stores = 0;
     int iter = 0;
     bool ok = true;
     for (int w = pair; w < total_work && ok; w += npairs, ++iter) {
@@ -611,7 +712,8 @@ mp_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a,
       if (!ptx::mbar_wait(&bars->tmem_full[acc], acc_phase)) { ok = false; break; }
       ptx::tc_fence_after_sync();
       const uint32_t bad =
-          epilogue_tile(p, tmem_base + acc * BN + ((uint32_t)(q * 32) << 16), row, n0, split, c_begin,
+          epilogue_tile<WIDE>(p, &map_out, stage, nslots, stores,
+                        tmem_base + acc * BN + ((uint32_t)(q * 32) << 16), row, n0, split, c_begin,
                         c_count, masked ? pass_bits : nullptr);
       if (p.out_mode == OUT_F16_FLAG && p.flag != nullptr) {
         if (__any_sync(0xFFFFFFFFu, bad != 0) && lane == 0) atomicOr(p.flag, 1);
@@ -622,6 +724,7 @@ mp_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a,
         ptx::mbar_arrive_cluster(ptx::map_to_cta(ptx::smem_u32(&bars->tmem_empty[acc]), 0));
     }
     if (!ok) report_timeout(bars);
+    if (lane == 0) ptx::bulk_wait_group_all();   // this warp's output stores have left shared memory
   }
 
   // ---------------------------------------------------------------- teardown
@@ -750,18 +853,18 @@ struct Operand {
   int64_t mn, red;    // extents along the output dimension and the reduction
 };
 
-template <bool A_MN, bool B_MN>
-int launch(const CUtensorMap& ma, const CUtensorMap& mb, const GemmParams& p, int grid,
-           cudaStream_t st) {
+template <bool A_MN, bool B_MN, bool WIDE>
+int launch(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mo, const GemmParams& p,
+           int grid, cudaStream_t st) {
   static bool attr_set = false;
   if (!attr_set) {
-    MP_CUDA_TRY(cudaFuncSetAttribute(mp_gemm_kernel<A_MN, B_MN>,
+    MP_CUDA_TRY(cudaFuncSetAttribute(mp_gemm_kernel<A_MN, B_MN, WIDE>,
                                      cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
     attr_set = true;
   }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(grid, 1, 1);
-  cfg.blockDim = dim3((p.bias != nullptr || p.act != 0) ? THREADS_FUSED : THREADS_PLAIN, 1, 1);
+  cfg.blockDim = dim3(WIDE ? THREADS_FUSED : THREADS_PLAIN, 1, 1);
   cfg.dynamicSmemBytes = SMEM_BYTES;
   cfg.stream = st;
   cudaLaunchAttribute attr;
@@ -769,21 +872,21 @@ int launch(const CUtensorMap& ma, const CUtensorMap& mb, const GemmParams& p, in
   attr.val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = &attr;
   cfg.numAttrs = 1;
-  MP_CUDA_TRY(cudaLaunchKernelEx(&cfg, mp_gemm_kernel<A_MN, B_MN>, ma, mb, p));
+  MP_CUDA_TRY(cudaLaunchKernelEx(&cfg, mp_gemm_kernel<A_MN, B_MN, WIDE>, ma, mb, mo, p));
   mp::count_launch();
   return MP_OK;
 }
 
-template <bool A_MN, bool B_MN>
+template <bool A_MN, bool B_MN, bool WIDE>
 int launch_pair(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mb32,
-                const GemmParams& p, int64_t work, cudaStream_t st) {
+                const CUtensorMap& mo, const GemmParams& p, int64_t work, cudaStream_t st) {
   static int max_pairs = 0;
   if (max_pairs == 0) {
-    MP_CUDA_TRY(cudaFuncSetAttribute(mp_gemm_pair_kernel<A_MN, B_MN>,
+    MP_CUDA_TRY(cudaFuncSetAttribute(mp_gemm_pair_kernel<A_MN, B_MN, WIDE>,
                                      cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM2_BYTES));
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2 * kModelSMs, 1, 1);
-    cfg.blockDim = dim3(THREADS, 1, 1);
+    cfg.blockDim = dim3(WIDE ? THREADS_FUSED : THREADS_PLAIN, 1, 1);
     cfg.dynamicSmemBytes = SMEM2_BYTES;
     cudaLaunchAttribute attr;
     attr.id = cudaLaunchAttributeClusterDimension;
@@ -791,14 +894,14 @@ int launch_pair(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap&
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
     int n = 0;
-    MP_CUDA_TRY(cudaOccupancyMaxActiveClusters(&n, mp_gemm_pair_kernel<A_MN, B_MN>, &cfg));
+    MP_CUDA_TRY(cudaOccupancyMaxActiveClusters(&n, mp_gemm_pair_kernel<A_MN, B_MN, WIDE>, &cfg));
     if (n < 1) return mp::set_error(MP_ERR_CUDA, "no CTA pair of the GEMM kernel fits on this device");
     max_pairs = n;
   }
   const int pairs = (int)(work < max_pairs ? work : max_pairs);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(2 * pairs, 1, 1);
-  cfg.blockDim = dim3((p.bias != nullptr || p.act != 0) ? THREADS_FUSED : THREADS_PLAIN, 1, 1);
+  cfg.blockDim = dim3(WIDE ? THREADS_FUSED : THREADS_PLAIN, 1, 1);
   cfg.dynamicSmemBytes = SMEM2_BYTES;
   cfg.stream = st;
   cudaLaunchAttribute attr;
@@ -806,7 +909,7 @@ int launch_pair(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap&
   attr.val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = &attr;
   cfg.numAttrs = 1;
-  MP_CUDA_TRY(cudaLaunchKernelEx(&cfg, mp_gemm_pair_kernel<A_MN, B_MN>, ma, mb, mb32, p));
+  MP_CUDA_TRY(cudaLaunchKernelEx(&cfg, mp_gemm_pair_kernel<A_MN, B_MN, WIDE>, ma, mb, mb32, mo, p));
   mp::count_launch();
   return MP_OK;
 }
@@ -831,8 +934,9 @@ int run_gemm(const char* name, const Operand& A, const Operand& B, void* out, in
   if (int rc = mp::check_device()) return rc;
   if (int rc = load_encoder()) return rc;
 
+  const int64_t No8 = No & ~(int64_t)7;
   GemmParams p;
-  p.Mo = (int)Mo; p.No = (int)No; p.R = (int)R;
+  p.Mo = (int)Mo; p.No = (int)No; p.R = (int)R; p.No8 = (int)No8;
   const bool pair = use_pair_kernel(Mo);
   p.m_tiles = (int)(pair ? (Mo + 255) / 256 : (Mo + BM - 1) / BM);
   p.n_tiles = (int)((No + BN - 1) / BN);
@@ -852,7 +956,10 @@ int run_gemm(const char* name, const Operand& A, const Operand& B, void* out, in
                            workspace ? ws_bytes : (size_t)0);
   }
 
-  CUtensorMap ma, mb, mb32;
+  CUtensorMap ma, mb, mb32, mo;
+  // FP16 output: 32-row x 64-column boxes, the unit one epilogue warp stores at a time
+  // (first No8 columns; a map over 8 columns that is never used when No < 8)
+  if (int rc = make_map(&mo, out, No8 > 0 ? No8 : 8, Mo, ldo, 64, 32)) return rc;
   if (int rc = A.mn_major ? make_map(&ma, A.ptr, A.mn, A.red, A.ld, 64, BK)
                           : make_map(&ma, A.ptr, A.red, A.mn, A.ld, BK, BM)) return rc;
   if (int rc = B.mn_major ? make_map(&mb, B.ptr, B.mn, B.red, B.ld, 64, BK)
@@ -870,18 +977,19 @@ int run_gemm(const char* name, const Operand& A, const Operand& B, void* out, in
   const int64_t work = (int64_t)p.m_tiles * p.n_tiles * p.splits;
   const int grid = (int)(work < sms ? work : sms);
 
+  // eight epilogue warps (two per scheduler) for the bias / activation / mask flavours, four for
+  // the plain ones
   int rc;
-  if (pair) {
-    if (A.mn_major && B.mn_major) rc = launch_pair<true, true>(ma, mb, mb32, p, work, st);
-    else if (!A.mn_major && B.mn_major) rc = launch_pair<false, true>(ma, mb, mb32, p, work, st);
-    else if (!A.mn_major && !B.mn_major) rc = launch_pair<false, false>(ma, mb, mb32, p, work, st);
-    else rc = launch_pair<true, false>(ma, mb, mb32, p, work, st);
-  } else {
-    if (A.mn_major && B.mn_major) rc = launch<true, true>(ma, mb, p, grid, st);
-    else if (!A.mn_major && B.mn_major) rc = launch<false, true>(ma, mb, p, grid, st);
-    else if (!A.mn_major && !B.mn_major) rc = launch<false, false>(ma, mb, p, grid, st);
-    else rc = launch<true, false>(ma, mb, p, grid, st);
-  }
+#define MP_DISPATCH(FN, ...)                                                                   \
+  do {                                                                                         \
+    if (A.mn_major && B.mn_major) rc = fused ? FN<true, true, true>(__VA_ARGS__) : FN<true, true, false>(__VA_ARGS__); \
+    else if (!A.mn_major && B.mn_major) rc = fused ? FN<false, true, true>(__VA_ARGS__) : FN<false, true, false>(__VA_ARGS__); \
+    else if (!A.mn_major && !B.mn_major) rc = fused ? FN<false, false, true>(__VA_ARGS__) : FN<false, false, false>(__VA_ARGS__); \
+    else rc = fused ? FN<true, false, true>(__VA_ARGS__) : FN<true, false, false>(__VA_ARGS__); \
+  } while (0)
+  if (pair) MP_DISPATCH(launch_pair, ma, mb, mb32, mo, p, work, st);
+  else MP_DISPATCH(launch, ma, mb, mo, p, grid, st);
+#undef MP_DISPATCH
   if (rc) return rc;
 
   if (p.splits > 1) {

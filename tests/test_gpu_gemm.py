@@ -12,17 +12,23 @@ def _pad8(n):
 
 def _to_dev(bits: np.ndarray):
     """uint16 bit patterns [R,C] -> CUDA FP16 view [R,C] inside a buffer whose row pitch is a
-    multiple of 8 elements (the library's alignment rule)."""
+    multiple of 8 elements (the library's alignment rule).  The padding columns hold NaN: an
+    operand element read from beyond the view would poison the result."""
     r, c = bits.shape
-    buf = torch.zeros(r, _pad8(c), dtype=torch.float16, device="cuda")
+    buf = torch.full((r, _pad8(c)), float("nan"), dtype=torch.float16, device="cuda")
     buf[:, :c] = torch.from_numpy(bits.view(np.float16)).cuda()
     return buf[:, :c]
 
 
+GUARD_ROWS = 3
+
+
 def _out(r, c, fill=0x5A5A):
-    buf = torch.full((r, _pad8(c)), 0, dtype=torch.int16, device="cuda")
+    """Output view [r, c] inside a pattern-filled buffer with padding columns and guard rows
+    before and after: whatever the kernel writes outside the view shows up."""
+    buf = torch.full((r + 2 * GUARD_ROWS, _pad8(c) + 8), 0, dtype=torch.int16, device="cuda")
     buf.fill_(fill if fill < 0x8000 else fill - 0x10000)
-    return buf.view(torch.float16)[:, :c], buf
+    return buf.view(torch.float16)[GUARD_ROWS:GUARD_ROWS + r, :c], buf
 
 
 def _bits(t):
@@ -51,9 +57,9 @@ def _run(mp, op, A, B, state=None):
         mp.mp_linear_bwd_wgrad(dA, dB, out, state, ws)
     torch.cuda.synchronize()
     assert mp.mp_gemm_device_status() == 0
-    # padding columns of the output buffer must be untouched
-    pad = raw[:, out.shape[1]:]
-    assert bool((pad == 0x5A5A).all())
+    # padding columns and guard rows of the output buffer must be untouched
+    assert bool((raw[:, out.shape[1]:] == 0x5A5A).all())
+    assert bool((raw[:GUARD_ROWS] == 0x5A5A).all()) and bool((raw[-GUARD_ROWS:] == 0x5A5A).all())
     return _bits(out), ws_bytes
 
 
