@@ -286,38 +286,46 @@ __device__ __forceinline__ void finish_group(const GemmParams& p, const CUtensor
 // instruction stream matters more to it than anything else.
 template <bool FUSED>
 __device__ __forceinline__ uint32_t epilogue_tile(const GemmParams& p, const CUtensorMap* map_out,
-                                                  uint8_t* stage, int nslots, int& stores,
+                                                  const CUtensorMap* map_ws, uint8_t* stage, int nslots,
+                                                  int& stores,
                                                   uint32_t tmem_acc, int row, int n0, int split,
                                                   int c_begin, int c_count,
                                                   const uint32_t* pass_bits = nullptr) {
   const bool row_ok = row < p.Mo;
   const int lane = threadIdx.x & 31;
+  if (row - lane >= p.Mo) return 0;             // nothing of this warp's rows exists
   if (p.out_mode == OUT_PARTIAL) {
-    // FP32 partial sums of a split reduction: 128 contiguous bytes per thread and chunk
+    // FP32 partial sums of a split reduction: a chunk (32 rows x 32 floats = 4 KiB) fills one
+    // staging slot; the workspace map is [split][row][column], so rows beyond Mo are clipped
+    // instead of landing in the next split's plane (its padded row length is a multiple of 4
+    // floats, so the 16-byte clipping of the columns is exact)
 #pragma unroll 1
     for (int c = c_begin; c < c_begin + c_count; ++c) {
       const int col0 = n0 + c * 32;
       if (col0 >= p.No) break;                  // warp-uniform
+      uint8_t* slot = stage + (stores % nslots) * SLOT_BYTES;
+      if (lane == 0) {
+        if (nslots == 2) ptx::bulk_wait_group_read<1>(); else ptx::bulk_wait_group_read<0>();
+      }
+      __syncwarp();
       uint32_t r[32];
       ptx::tmem_ld_32x32(tmem_acc + c * 32, r);
       ptx::tmem_ld_wait();
-      if (row_ok) {
-        float* dst = p.ws + ((int64_t)split * p.Mo + row) * p.ws_ld + col0;
-        if (col0 + 32 <= p.No) {
+      uint8_t* rowp = slot + lane * 128;
 #pragma unroll
-          for (int j = 0; j < 8; ++j)
-            *reinterpret_cast<uint4*>(dst + 4 * j) =
-                make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
-        } else {
-#pragma unroll
-          for (int j = 0; j < 32; ++j)
-            if (col0 + j < p.No) dst[j] = __uint_as_float(r[j]);
-        }
+      for (int j = 0; j < 8; ++j)
+        *reinterpret_cast<uint4*>(rowp + ((j ^ (lane & 7)) << 4)) =
+            make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
+      ptx::fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) {
+        ptx::tma_store_3d(map_ws, slot, col0, row - lane, split);
+        ptx::bulk_commit_group();
       }
+      ++stores;
     }
     return 0;
   }
-  if (row - lane >= p.Mo) return 0;             // nothing of this warp's rows exists
   uint32_t flag_acc = 0;
   // groups of 64 columns g_begin .. g_end that have columns (warp-uniform)
   const int g_begin = c_begin >> 1;
@@ -341,7 +349,8 @@ __device__ __forceinline__ uint32_t epilogue_tile(const GemmParams& p, const CUt
 template <bool A_MN, bool B_MN, bool WIDE>
 __global__ void __launch_bounds__(WIDE ? THREADS_FUSED : THREADS_PLAIN, 1)
 mp_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-               const __grid_constant__ CUtensorMap map_out, const GemmParams p) {
+               const __grid_constant__ CUtensorMap map_out, const __grid_constant__ CUtensorMap map_ws,
+               const GemmParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                              ~static_cast<uintptr_t>(1023));
@@ -494,7 +503,7 @@ mp_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       if (masked) load_pass_bits(p, row, n0, c_begin, c_count, pass_bits);   // runs under the tile's main loop
       if (!ptx::mbar_wait(&bars->tmem_full[acc], acc_phase)) { ok = false; break; }
       ptx::tc_fence_after_sync();
-      const uint32_t bad = epilogue_tile<WIDE>(p, &map_out, stage, nslots, stores,
+      const uint32_t bad = epilogue_tile<WIDE>(p, &map_out, &map_ws, stage, nslots, stores,
                                          tmem_base + acc * BN + ((uint32_t)(q * 32) << 16), row, n0, split,
                                          c_begin, c_count, masked ? pass_bits : nullptr);
       if (p.out_mode == OUT_F16_FLAG && p.flag != nullptr) {
@@ -542,7 +551,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(WIDE ? THREADS_FUSED
 mp_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a,
                     const __grid_constant__ CUtensorMap map_b,
                     const __grid_constant__ CUtensorMap map_b32,
-                    const __grid_constant__ CUtensorMap map_out, const GemmParams p) {
+                    const __grid_constant__ CUtensorMap map_out,
+                    const __grid_constant__ CUtensorMap map_ws, const GemmParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                              ~static_cast<uintptr_t>(1023));
@@ -712,7 +722,7 @@ mp_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a,
       if (!ptx::mbar_wait(&bars->tmem_full[acc], acc_phase)) { ok = false; break; }
       ptx::tc_fence_after_sync();
       const uint32_t bad =
-          epilogue_tile<WIDE>(p, &map_out, stage, nslots, stores,
+          epilogue_tile<WIDE>(p, &map_out, &map_ws, stage, nslots, stores,
                         tmem_base + acc * BN + ((uint32_t)(q * 32) << 16), row, n0, split, c_begin,
                         c_count, masked ? pass_bits : nullptr);
       if (p.out_mode == OUT_F16_FLAG && p.flag != nullptr) {
@@ -756,7 +766,18 @@ mp_splitk_reduce_kernel(const float* __restrict__ ws, int splits, int Mo, int No
     const float* src = ws + (int64_t)row * ws_ld + col;
     if (col + 4 <= No) {
       float4 acc = *reinterpret_cast<const float4*>(src);
-      for (int s = 1; s < splits; ++s) {
+      int s = 1;
+      for (; s + 3 < splits; s += 4) {            // four loads in flight, added in ascending order
+        float4 x[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) x[u] = *reinterpret_cast<const float4*>(src + (s + u) * split_stride);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          acc.x = __fadd_rn(acc.x, x[u].x); acc.y = __fadd_rn(acc.y, x[u].y);
+          acc.z = __fadd_rn(acc.z, x[u].z); acc.w = __fadd_rn(acc.w, x[u].w);
+        }
+      }
+      for (; s < splits; ++s) {
         const float4 x = *reinterpret_cast<const float4*>(src + s * split_stride);
         acc.x = __fadd_rn(acc.x, x.x); acc.y = __fadd_rn(acc.y, x.y);
         acc.z = __fadd_rn(acc.z, x.z); acc.w = __fadd_rn(acc.w, x.w);
@@ -810,6 +831,22 @@ int make_map(CUtensorMap* map, const void* ptr, int64_t inner, int64_t outer, in
   return MP_OK;
 }
 
+// 3-D FP32 tensor map over the split-reduction workspace: `ld` floats per row (a multiple of 4),
+// `rows` rows per split, `splits` planes; one box is 32 floats x 32 rows of one plane.
+int make_map_ws(CUtensorMap* map, const void* ptr, int64_t ld, int64_t rows, int64_t splits) {
+  const cuuint64_t dims[3] = {(cuuint64_t)ld, (cuuint64_t)rows, (cuuint64_t)splits};
+  const cuuint64_t strides[2] = {(cuuint64_t)ld * 4, (cuuint64_t)rows * (cuuint64_t)ld * 4};
+  const cuuint32_t box[3] = {32, 32, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  const CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void*>(ptr), dims,
+                              strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS)
+    return mp::set_error(MP_ERR_CUDA, "cuTensorMapEncodeTiled (workspace) failed with code %d", (int)r);
+  return MP_OK;
+}
+
 // Number of reduction splits: minimise a simple time model (waves of tiles on the SMs plus
 // the workspace round trip).  Depends only on the sizes, so that the workspace query and the
 // launch always agree.
@@ -854,8 +891,8 @@ struct Operand {
 };
 
 template <bool A_MN, bool B_MN, bool WIDE>
-int launch(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mo, const GemmParams& p,
-           int grid, cudaStream_t st) {
+int launch(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mo, const CUtensorMap& mw,
+           const GemmParams& p, int grid, cudaStream_t st) {
   static bool attr_set = false;
   if (!attr_set) {
     MP_CUDA_TRY(cudaFuncSetAttribute(mp_gemm_kernel<A_MN, B_MN, WIDE>,
@@ -872,14 +909,15 @@ int launch(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mo, 
   attr.val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = &attr;
   cfg.numAttrs = 1;
-  MP_CUDA_TRY(cudaLaunchKernelEx(&cfg, mp_gemm_kernel<A_MN, B_MN, WIDE>, ma, mb, mo, p));
+  MP_CUDA_TRY(cudaLaunchKernelEx(&cfg, mp_gemm_kernel<A_MN, B_MN, WIDE>, ma, mb, mo, mw, p));
   mp::count_launch();
   return MP_OK;
 }
 
 template <bool A_MN, bool B_MN, bool WIDE>
 int launch_pair(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mb32,
-                const CUtensorMap& mo, const GemmParams& p, int64_t work, cudaStream_t st) {
+                const CUtensorMap& mo, const CUtensorMap& mw, const GemmParams& p, int64_t work,
+                cudaStream_t st) {
   static int max_pairs = 0;
   if (max_pairs == 0) {
     MP_CUDA_TRY(cudaFuncSetAttribute(mp_gemm_pair_kernel<A_MN, B_MN, WIDE>,
@@ -909,7 +947,7 @@ int launch_pair(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap&
   attr.val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = &attr;
   cfg.numAttrs = 1;
-  MP_CUDA_TRY(cudaLaunchKernelEx(&cfg, mp_gemm_pair_kernel<A_MN, B_MN, WIDE>, ma, mb, mb32, mo, p));
+  MP_CUDA_TRY(cudaLaunchKernelEx(&cfg, mp_gemm_pair_kernel<A_MN, B_MN, WIDE>, ma, mb, mb32, mo, mw, p));
   mp::count_launch();
   return MP_OK;
 }
@@ -956,7 +994,7 @@ int run_gemm(const char* name, const Operand& A, const Operand& B, void* out, in
                            workspace ? ws_bytes : (size_t)0);
   }
 
-  CUtensorMap ma, mb, mb32, mo;
+  CUtensorMap ma, mb, mb32, mo, mw;
   // FP16 output: 32-row x 64-column boxes, the unit one epilogue warp stores at a time
   // (first No8 columns; a map over 8 columns that is never used when No < 8)
   if (int rc = make_map(&mo, out, No8 > 0 ? No8 : 8, Mo, ldo, 64, 32)) return rc;
@@ -969,6 +1007,13 @@ int run_gemm(const char* name, const Operand& A, const Operand& B, void* out, in
     if (int rc = make_map(&mb32, B.ptr, B.red, B.mn, B.ld, BK, 32)) return rc;
   } else {
     mb32 = mb;
+  }
+
+  // FP32 partial sums of a split reduction: [split][row][padded column], boxes of 32 x 32 floats
+  if (p.splits > 1) {
+    if (int rc = make_map_ws(&mw, workspace, p.ws_ld, Mo, p.splits)) return rc;
+  } else {
+    mw = mo;
   }
 
   int dev = 0, sms = 0;
@@ -987,8 +1032,8 @@ int run_gemm(const char* name, const Operand& A, const Operand& B, void* out, in
     else if (!A.mn_major && !B.mn_major) rc = fused ? FN<false, false, true>(__VA_ARGS__) : FN<false, false, false>(__VA_ARGS__); \
     else rc = fused ? FN<true, false, true>(__VA_ARGS__) : FN<true, false, false>(__VA_ARGS__); \
   } while (0)
-  if (pair) MP_DISPATCH(launch_pair, ma, mb, mb32, mo, p, work, st);
-  else MP_DISPATCH(launch, ma, mb, mo, p, grid, st);
+  if (pair) MP_DISPATCH(launch_pair, ma, mb, mb32, mo, mw, p, work, st);
+  else MP_DISPATCH(launch, ma, mb, mo, mw, p, grid, st);
 #undef MP_DISPATCH
   if (rc) return rc;
 
