@@ -371,6 +371,10 @@ def main():
             stack.load_weights(l, w, w.half())
     gen.manual_seed(99 + rank)                 # each rank its own rows
     xs, gs, xs_host, gs_host = [], [], [], []
+    # the FP32 gradients entering the top layers arrive as slices of one flat buffer
+    tops = [l for l in range(L) if not stack.feeds_next(l)]
+    g_flat = torch.empty(sum(cfg.shapes[l][0] * cfg.shapes[l][2] for l in tops), device="cuda")
+    g_off = 0
     for l, (M, K, N) in enumerate(cfg.shapes):
         if chained[l]:
             xs.append(None); xs_host.append(None)
@@ -385,7 +389,9 @@ def main():
         if stack.feeds_next(l):
             gs.append(None); gs_host.append(None)
         else:
-            g = torch.randn(M, N, generator=gen, device="cuda") * cfg.grad_std
+            g = g_flat[g_off:g_off + M * N].view(M, N)
+            g_off += M * N
+            g.copy_(torch.randn(M, N, generator=gen, device="cuda") * cfg.grad_std)
             gs.append(g)
             gs_host.append(g.cpu().pin_memory())
     h2d = sum(t.numel() * t.element_size() for t in xs_host + gs_host if t is not None)

@@ -81,11 +81,28 @@ class LinearStack:
         self.y = [torch.empty(m, _align(n), **f16) for m, _, n in self.shapes]
         self.dy = [None] * self.L
         self.dx = [torch.empty(m, _align(k), **f16) for m, k, _ in self.shapes]
+        # Scaled upstream gradients of the top layers whose rows need no padding share one flat
+        # buffer (ascending layer order): when their FP32 gradients arrive as consecutive slices
+        # of one buffer too, a single scaling call covers all of them.
+        self.flat_tops = [l for l in range(self.L) if not (l + 1 < self.L and self.chained[l + 1])
+                          and self.shapes[l][2] % 8 == 0]
+        self.dy_top_flat = torch.zeros(sum(self.shapes[l][0] * self.shapes[l][2] for l in self.flat_tops), **f16)
+        flat_off = {}
+        o = 0
+        for l in self.flat_tops:
+            flat_off[l] = o
+            o += self.shapes[l][0] * self.shapes[l][2]
         for l in range(self.L):
             if self.chained[l]:
                 self.x[l] = self.y[l - 1]
             feeds = l + 1 < self.L and self.chained[l + 1]
-            self.dy[l] = self.dx[l + 1] if feeds else torch.zeros(self.shapes[l][0], _align(self.shapes[l][2]), **f16)
+            if feeds:
+                self.dy[l] = self.dx[l + 1]
+            elif l in flat_off:
+                m, _, n = self.shapes[l]
+                self.dy[l] = self.dy_top_flat[flat_off[l]:flat_off[l] + m * n].view(m, n)
+            else:
+                self.dy[l] = torch.zeros(self.shapes[l][0], _align(self.shapes[l][2]), **f16)
         need = 0
         for m, k, n in self.shapes:
             for op in (mp.MP_OP_FWD, mp.MP_OP_DGRAD, mp.MP_OP_WGRAD):
@@ -229,6 +246,24 @@ class LinearStack:
     _host_graph = None
     use_graph_from_host = False
 
+    def _flat_upstream(self, gs):
+        """The FP32 gradients of the flat top layers as one tensor, if they are consecutive
+        contiguous slices of one buffer in ascending layer order; else None."""
+        ls = self.flat_tops
+        if len(ls) < 2 or any(gs[l] is None for l in ls):
+            return None
+        first = gs[ls[0]]
+        store, off = first.untyped_storage(), first.storage_offset()
+        for l in ls:
+            t = gs[l]
+            if (t.dtype != torch.float32 or not t.is_contiguous() or t.storage_offset() != off
+                    or t.untyped_storage().data_ptr() != store.data_ptr()
+                    or t.numel() != self.shapes[l][0] * self.shapes[l][2]):
+                return None
+            off += t.numel()
+        return torch.empty(0, dtype=torch.float32, device=first.device).set_(
+            store, first.storage_offset(), (off - first.storage_offset(),))
+
     # ---- the step ----
     def step(self, xs, gs):
         """xs[l]: FP16 [M,K] CUDA tensor (row pitch a multiple of 8) for a layer that is not
@@ -243,8 +278,11 @@ class LinearStack:
             else:
                 self._call("fwd", mp.mp_linear_fwd_act, self.x[l][:, :self.shapes[l][1]], self.W16(l),
                            self.b16[l], self.Y(l), self.acts[l], self.clip, self.workspace)
+        g_flat = self._flat_upstream(gs)
+        if g_flat is not None:        # one scaling call for all flat top layers
+            self._call("scale", mp.mp_scale_upstream, g_flat, self.dy_top_flat, self.state)
         for l in range(self.L - 1, -1, -1):
-            if not self.feeds_next(l):
+            if not self.feeds_next(l) and not (g_flat is not None and l in self.flat_tops):
                 n = self.shapes[l][2]
                 if self.dy[l].shape[1] == n:
                     self._call("scale", mp.mp_scale_upstream, gs[l], self.dy[l], self.state)
@@ -293,10 +331,19 @@ class HostPipeline:
         self.copy_stream = torch.cuda.Stream(device=s.device)
         mk_x = lambda l: None if s.chained[l] else torch.zeros(
             s.shapes[l][0], _align(s.shapes[l][1]), dtype=torch.float16, device=s.device)
-        mk_g = lambda l: None if s.feeds_next(l) else torch.zeros(
-            s.shapes[l][0], s.shapes[l][2], dtype=torch.float32, device=s.device)
+
+        def mk_gs():      # one flat FP32 buffer, sliced per top layer: the step scales it in one call
+            tops = [l for l in range(s.L) if not s.feeds_next(l)]
+            flat = torch.zeros(sum(s.shapes[l][0] * s.shapes[l][2] for l in tops), dtype=torch.float32,
+                               device=s.device)
+            out, o = [None] * s.L, 0
+            for l in tops:
+                m, _, n = s.shapes[l]
+                out[l] = flat[o:o + m * n].view(m, n)
+                o += m * n
+            return out
         self.x_in = [[mk_x(l) for l in range(s.L)] for _ in range(2)]
-        self.g_in = [[mk_g(l) for l in range(s.L)] for _ in range(2)]
+        self.g_in = [mk_gs() for _ in range(2)]
         self.ready = [None, None]        # event: the set's copies have landed
         self.consumed = [None, None]     # event: the step that read the set has finished
         self.graphs = [None, None]

@@ -254,6 +254,46 @@ def test_graph_replay_equals_call_by_call(orc, mp):
     a.close(); b.close()
 
 
+def test_one_scaling_call_over_a_flat_gradient_buffer(orc, mp):
+    """When the FP32 gradients entering the top layers are consecutive slices of one buffer the
+    stack scales them with one call; the scaled gradients and the state after the steps are
+    bit-for-bit those of one call per layer, with fewer launches."""
+    from paper_1805_10387_b200.stack import LinearStack
+    shapes = [(96, 64, 40), (96, 40, 72), (96, 64, 72)]      # three independent layers
+    chained = [False, False, False]
+    rng = np.random.default_rng(11)
+    ws = [rng.standard_normal((k, n)).astype(np.float32) / np.sqrt(k) for _, k, n in shapes]
+
+    def make():
+        st = LinearStack(shapes, chained, lr=1e-3, init_scale=1024.0, growth_interval=2)
+        for l, w in enumerate(ws):
+            st.load_weights(l, torch.from_numpy(w).cuda(), torch.from_numpy(w).cuda().half())
+        return st
+    a, b = make(), make()
+    xs = [torch.from_numpy(rng.standard_normal((m, k)).astype(np.float32)).cuda().half() for m, k, _ in shapes]
+    g_sep = [torch.from_numpy((rng.standard_normal((m, n)) * 1e-3).astype(np.float32)).cuda() for m, _, n in shapes]
+    flat = torch.cat([g.reshape(-1) for g in g_sep])
+    g_flat, o = [], 0
+    for m, _, n in shapes:
+        g_flat.append(flat[o:o + m * n].view(m, n)); o += m * n
+    assert a._flat_upstream(g_sep) is None and b._flat_upstream(g_flat) is not None
+    n0 = mp.mp_kernel_launch_count()
+    for _ in range(3):
+        a.step(xs, g_sep)
+    n1 = mp.mp_kernel_launch_count()
+    for _ in range(3):
+        b.step(xs, g_flat)
+    n2 = mp.mp_kernel_launch_count()
+    torch.cuda.synchronize()
+    assert (n1 - n0) - (n2 - n1) == 3 * (len(shapes) - 1)
+    for l in range(len(shapes)):
+        assert torch.equal(a.dY(l).contiguous().view(torch.int16), b.dY(l).contiguous().view(torch.int16))
+    for fa, fb in ((a.w32_flat, b.w32_flat), (a.m_flat, b.m_flat), (a.v_flat, b.v_flat)):
+        assert torch.equal(fa.view(torch.int32), fb.view(torch.int32))
+    assert a.state.read().scale == b.state.read().scale
+    a.close(); b.close()
+
+
 def test_host_pipeline_equals_serial_host_steps(orc, mp):
     """Batches fed from pinned host memory through the double-buffered pipeline (copy of batch
     i+1 under the step of batch i, one CUDA graph per staging set) leave bit-for-bit the state
