@@ -168,6 +168,31 @@ int mp_linear_bwd_wgrad_static(const void* X16, int64_t ldx, const void* dY16, i
 /* Size of that built-in scratch in bytes (equals MP_STATIC_SCRATCH_BYTES). */
 size_t mp_static_scratch_bytes(void);
 
+/* ---- several independent layers of one shape in one launch ------------------------------
+ * The products of Section 3.1 for `count` (1 .. mp_max_group()) layers that have the same M, K,
+ * N and leading dimensions and do not depend on one another (the query, key and value
+ * projections of an attention block; the per-layer gate products of a stack whose layers are
+ * fed independently).  X16, W16, Y16 ... are host arrays of `count` device pointers; each
+ * problem obeys the rules of the single call of the same name and gets that call's result (bit
+ * for bit when both split the reduction the same way; otherwise the FP32 partial sums are added
+ * in another, equally fixed order).  One launch walks the tiles of all problems, so a product too small to fill
+ * the GPU's waves on its own does not leave SMs idle.  workspace: at least
+ * mp_gemm_workspace_bytes_grouped(count, M, K, N, op) bytes.  Errors as for the single calls;
+ * INVALID_ARG also for count outside 1 .. mp_max_group(). */
+int mp_linear_fwd_grouped(int count, const void* const* X16, int64_t ldx, const void* const* W16,
+                          int64_t ldw, void* const* Y16, int64_t ldy, int64_t M, int64_t K, int64_t N,
+                          void* workspace, size_t workspace_bytes, void* stream);
+int mp_linear_bwd_dgrad_grouped(int count, const void* const* dY16, int64_t lddy, const void* const* W16,
+                                int64_t ldw, void* const* dX16, int64_t lddx, int64_t M, int64_t K,
+                                int64_t N, void* workspace, size_t workspace_bytes, void* stream);
+/* ORs "an inf or NaN was stored" of every problem into state->found_inf (state may be NULL). */
+int mp_linear_bwd_wgrad_grouped(int count, const void* const* X16, int64_t ldx, const void* const* dY16,
+                                int64_t lddy, void* const* dW16, int64_t lddw, int64_t M, int64_t K,
+                                int64_t N, mp_state* state, void* workspace, size_t workspace_bytes,
+                                void* stream);
+/* Largest `count` the grouped calls take. */
+int mp_max_group(void);
+
 /* ---- layers with a bias and an activation ------------------------------------------------
  * The models of the paper's Section 5 follow their dense products with a bias and a
  * nonlinearity (ReLU in the Transformer feed-forward block, clipped ReLU in DeepSpeech2).  The
@@ -223,6 +248,8 @@ enum { MP_OP_FWD = 0, MP_OP_DGRAD = 1, MP_OP_WGRAD = 2 };
 
 /* Scratch bytes the GEMM of `op` needs for these sizes (0 when it needs none). */
 size_t mp_gemm_workspace_bytes(int64_t M, int64_t K, int64_t N, int op);
+/* The same for a grouped call over `count` problems (0 for a count the calls refuse). */
+size_t mp_gemm_workspace_bytes_grouped(int count, int64_t M, int64_t K, int64_t N, int op);
 
 /* dY16[i] = rn16( S * g32[i] ), S read from the device state (Section 3.1, item 1: the loss
  * is scaled; for a linear stack that is the gradient entering the top layer). */

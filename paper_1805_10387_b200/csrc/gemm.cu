@@ -56,14 +56,23 @@ __device__ int g_gemm_status = 0;              // first device-side error (bound
 
 enum OutMode { OUT_F16 = 0, OUT_F16_FLAG = 1, OUT_PARTIAL = 2 };
 
+// Up to MAX_GROUP independent products of the same shape and layouts run as one launch: the
+// work list is problem-major, and every role picks its tensor maps by problem index.
+constexpr int MAX_GROUP = 4;
+struct GroupMaps {
+  CUtensorMap a[MAX_GROUP], b[MAX_GROUP], b32[MAX_GROUP], out[MAX_GROUP], ws[MAX_GROUP];
+};
+
 struct GemmParams {
+  int group;            // number of problems in this launch
+  int work_per_problem; // tiles x splits of one problem
   int Mo, No, R;        // output rows, output columns, reduction length
   int No8;              // No rounded down to a multiple of 8: the columns the output tensor map covers
   int m_tiles, n_tiles, splits, num_kb;
   int out_mode;
-  uint16_t* out;        // FP16 output [Mo, No], leading dimension ldo
+  uint16_t* out[MAX_GROUP];   // FP16 outputs [Mo, No], leading dimension ldo
   int64_t ldo;
-  float* ws;            // FP32 partials [splits][Mo][ws_ld]
+  float* ws;            // FP32 partials [problem][splits][Mo][ws_ld]
   int64_t ws_ld;
   int* flag;            // found_inf word, or null
   // Optional fused epilogue (FP16 output only).  Forward flavour: add bias[col] to the FP32 sum,
@@ -173,7 +182,8 @@ constexpr int SLOT_BYTES = 32 * 64 * 2;
 template <bool FUSED>
 __device__ __forceinline__ void finish_chunk(const GemmParams& p, uint32_t (&r)[32], int col0, int row,
                                              bool row_ok, int lane, uint8_t* slot, int half,
-                                             const uint32_t* pass_bits, int c, uint32_t& flag_acc) {
+                                             const uint32_t* pass_bits, int c, uint32_t& flag_acc,
+                                             int prob) {
   if (FUSED && (p.bias != nullptr || (p.act != 0 && p.mask == nullptr))) {
     // forward flavour, on the FP32 values: + bias, then the activation
     uint32_t bw[16];                          // 32 bias values as packed halves (0 if absent)
@@ -232,7 +242,7 @@ __device__ __forceinline__ void finish_chunk(const GemmParams& p, uint32_t (&r)[
       for (int j = 0; j < 16; ++j) flag_acc |= (h[j] & 0x7C007C00u) + 0x04000400u;
     }
     if (col0 + 32 > p.No8) {                  // the columns past the tensor map's last 16-byte unit
-      uint16_t* dst = p.out + (int64_t)row * p.ldo + col0;
+      uint16_t* dst = p.out[prob] + (int64_t)row * p.ldo + col0;
 #pragma unroll
       for (int j = 0; j < 32; ++j)
         if (col0 + j >= p.No8 && col0 + j < p.No)
@@ -257,15 +267,16 @@ template <bool FUSED>
 __device__ __forceinline__ void finish_group(const GemmParams& p, const CUtensorMap* map_out, uint8_t* stage,
                                              int nslots, int& stores, uint32_t (&ra)[32], uint32_t (&rb)[32],
                                              bool second, int colg, int g, int row, bool row_ok, int lane,
-                                             const uint32_t* pass_bits, uint32_t& flag_acc) {
+                                             const uint32_t* pass_bits, uint32_t& flag_acc, int prob) {
   uint8_t* slot = stage + (stores % nslots) * SLOT_BYTES;
   // the slot must no longer be read by an earlier store
   if (lane == 0) {
     if (nslots == 2) ptx::bulk_wait_group_read<1>(); else ptx::bulk_wait_group_read<0>();
   }
   __syncwarp();
-  finish_chunk<FUSED>(p, ra, colg, row, row_ok, lane, slot, 0, pass_bits, 2 * g, flag_acc);
-  if (second) finish_chunk<FUSED>(p, rb, colg + 32, row, row_ok, lane, slot, 1, pass_bits, 2 * g + 1, flag_acc);
+  finish_chunk<FUSED>(p, ra, colg, row, row_ok, lane, slot, 0, pass_bits, 2 * g, flag_acc, prob);
+  if (second)
+    finish_chunk<FUSED>(p, rb, colg + 32, row, row_ok, lane, slot, 1, pass_bits, 2 * g + 1, flag_acc, prob);
   ptx::fence_proxy_async_smem();                // the slot is complete: hand it to the TMA unit
   __syncwarp();
   if (colg < p.No8) {                           // else: only register-stored columns in this group
@@ -289,7 +300,7 @@ __device__ __forceinline__ uint32_t epilogue_tile(const GemmParams& p, const CUt
                                                   const CUtensorMap* map_ws, uint8_t* stage, int nslots,
                                                   int& stores,
                                                   uint32_t tmem_acc, int row, int n0, int split,
-                                                  int c_begin, int c_count,
+                                                  int c_begin, int c_count, int prob,
                                                   const uint32_t* pass_bits = nullptr) {
   const bool row_ok = row < p.Mo;
   const int lane = threadIdx.x & 31;
@@ -341,16 +352,14 @@ __device__ __forceinline__ uint32_t epilogue_tile(const GemmParams& p, const CUt
     if (second) ptx::tmem_ld_32x32(tmem_acc + g * 64 + 32, rb);
     ptx::tmem_ld_wait();
     finish_group<FUSED>(p, map_out, stage, nslots, stores, ra, rb, second, colg, g, row, row_ok, lane,
-                        pass_bits, flag_acc);
+                        pass_bits, flag_acc, prob);
   }
   return flag_acc & 0x80008000u;
 }
 
 template <bool A_MN, bool B_MN, bool WIDE>
 __global__ void __launch_bounds__(WIDE ? THREADS_FUSED : THREADS_PLAIN, 1)
-mp_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-               const __grid_constant__ CUtensorMap map_out, const __grid_constant__ CUtensorMap map_ws,
-               const GemmParams p) {
+mp_gemm_kernel(const __grid_constant__ GroupMaps maps, const GemmParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                              ~static_cast<uintptr_t>(1023));
@@ -370,9 +379,9 @@ mp_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     }
     bars->abort = 0;
     ptx::fence_mbar_init();
-    ptx::prefetch_tensormap(&map_a);
-    ptx::prefetch_tensormap(&map_b);
-    ptx::prefetch_tensormap(&map_out);
+    ptx::prefetch_tensormap(&maps.a[0]);
+    ptx::prefetch_tensormap(&maps.b[0]);
+    ptx::prefetch_tensormap(&maps.out[0]);
   }
   if (warp == 1) {
     ptx::tmem_alloc(&bars->tmem_base, TMEM_COLS);
@@ -386,7 +395,7 @@ mp_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   // previous kernel in the stream; nothing below may.
   ptx::grid_dependency_wait();
 
-  const int total_work = p.m_tiles * p.n_tiles * p.splits;
+  const int total_work = p.group * p.work_per_problem;
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
@@ -395,7 +404,10 @@ mp_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     int issued = 0;
     bool ok = true;
     for (int w = blockIdx.x; w < total_work && ok; w += gridDim.x) {
-      const int split = w % p.splits, tile = w / p.splits;
+      const int prob = w / p.work_per_problem, wl = w - prob * p.work_per_problem;
+      const int split = wl % p.splits, tile = wl / p.splits;
+      const CUtensorMap* map_a = &maps.a[prob];
+      const CUtensorMap* map_b = &maps.b[prob];
       const int m0 = (tile / p.n_tiles) * BM, n0 = (tile % p.n_tiles) * BN;
       const int b_boxes = B_MN ? (tile_width(p.No, n0) + 63) / 64 : BN / 64;   // 64-column boxes of B
       const int kb0 = (int)((int64_t)split * p.num_kb / p.splits);
@@ -410,17 +422,17 @@ mp_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           if (A_MN) {
 #pragma unroll
             for (int c = 0; c < BM / 64; ++c)
-              ptx::tma_load_2d(sA + c * CHUNK_BYTES, &map_a, &bars->full[stage], m0 + 64 * c, k);
+              ptx::tma_load_2d(sA + c * CHUNK_BYTES, map_a, &bars->full[stage], m0 + 64 * c, k);
           } else {
-            ptx::tma_load_2d(sA, &map_a, &bars->full[stage], k, m0);
+            ptx::tma_load_2d(sA, map_a, &bars->full[stage], k, m0);
           }
           if (B_MN) {
 #pragma unroll
             for (int c = 0; c < BN / 64; ++c)
               if (c < b_boxes)
-                ptx::tma_load_2d(sB + c * CHUNK_BYTES, &map_b, &bars->full[stage], n0 + 64 * c, k);
+                ptx::tma_load_2d(sB + c * CHUNK_BYTES, map_b, &bars->full[stage], n0 + 64 * c, k);
           } else {
-            ptx::tma_load_2d(sB, &map_b, &bars->full[stage], k, n0);
+            ptx::tma_load_2d(sB, map_b, &bars->full[stage], k, n0);
           }
         }
         __syncwarp();
@@ -445,7 +457,8 @@ mp_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     int iter = 0;
     bool ok = true;
     for (int w = blockIdx.x; w < total_work && ok; w += gridDim.x, ++iter) {
-      const int split = w % p.splits, tile = w / p.splits;
+      const int wl = w % p.work_per_problem;
+      const int split = wl % p.splits, tile = wl / p.splits;
       const uint32_t idesc =
           ptx::idesc_f16_f32(BM, tile_width(p.No, (tile % p.n_tiles) * BN), A_MN, B_MN);
       const int kb0 = (int)((int64_t)split * p.num_kb / p.splits);
@@ -493,7 +506,8 @@ mp_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     int iter = 0;
     bool ok = true;
     for (int w = blockIdx.x; w < total_work && ok; w += gridDim.x, ++iter) {
-      const int split = w % p.splits, tile = w / p.splits;
+      const int prob = w / p.work_per_problem, wl = w - prob * p.work_per_problem;
+      const int split = wl % p.splits, tile = wl / p.splits;
       const int m0 = (tile / p.n_tiles) * BM, n0 = (tile % p.n_tiles) * BN;
       const int acc = iter & 1;
       const uint32_t acc_phase = (iter >> 1) & 1;
@@ -503,9 +517,9 @@ mp_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       if (masked) load_pass_bits(p, row, n0, c_begin, c_count, pass_bits);   // runs under the tile's main loop
       if (!ptx::mbar_wait(&bars->tmem_full[acc], acc_phase)) { ok = false; break; }
       ptx::tc_fence_after_sync();
-      const uint32_t bad = epilogue_tile<WIDE>(p, &map_out, &map_ws, stage, nslots, stores,
+      const uint32_t bad = epilogue_tile<WIDE>(p, &maps.out[prob], &maps.ws[prob], stage, nslots, stores,
                                          tmem_base + acc * BN + ((uint32_t)(q * 32) << 16), row, n0, split,
-                                         c_begin, c_count, masked ? pass_bits : nullptr);
+                                         c_begin, c_count, prob, masked ? pass_bits : nullptr);
       if (p.out_mode == OUT_F16_FLAG && p.flag != nullptr) {
         if (__any_sync(0xFFFFFFFFu, bad != 0) && lane == 0) atomicOr(p.flag, 1);
       }
@@ -548,11 +562,7 @@ struct Barriers2 {
 
 template <bool A_MN, bool B_MN, bool WIDE>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(WIDE ? THREADS_FUSED : THREADS_PLAIN, 1)
-mp_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a,
-                    const __grid_constant__ CUtensorMap map_b,
-                    const __grid_constant__ CUtensorMap map_b32,
-                    const __grid_constant__ CUtensorMap map_out,
-                    const __grid_constant__ CUtensorMap map_ws, const GemmParams p) {
+mp_gemm_pair_kernel(const __grid_constant__ GroupMaps maps, const GemmParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                              ~static_cast<uintptr_t>(1023));
@@ -574,10 +584,10 @@ mp_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a,
     }
     bars->abort = 0;
     ptx::fence_mbar_init();
-    ptx::prefetch_tensormap(&map_a);
-    ptx::prefetch_tensormap(&map_b);
-    if (!B_MN) ptx::prefetch_tensormap(&map_b32);
-    ptx::prefetch_tensormap(&map_out);
+    ptx::prefetch_tensormap(&maps.a[0]);
+    ptx::prefetch_tensormap(&maps.b[0]);
+    if (!B_MN) ptx::prefetch_tensormap(&maps.b32[0]);
+    ptx::prefetch_tensormap(&maps.out[0]);
   }
   if (warp == 1) {
     ptx::tmem_alloc_pair(&bars->tmem_base, TMEM_COLS);
@@ -592,7 +602,7 @@ mp_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a,
   ptx::grid_dependency_wait();
 
   const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
-  const int total_work = p.m_tiles * p.n_tiles * p.splits;   // m_tiles counts 256-row tiles here
+  const int total_work = p.group * p.work_per_problem;   // m_tiles counts 256-row tiles here
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer (both CTAs)
@@ -601,7 +611,11 @@ mp_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a,
     int issued = 0;
     bool ok = true;
     for (int w = pair; w < total_work && ok; w += npairs) {
-      const int split = w % p.splits, tile = w / p.splits;
+      const int prob = w / p.work_per_problem, wl = w - prob * p.work_per_problem;
+      const int split = wl % p.splits, tile = wl / p.splits;
+      const CUtensorMap* map_a = &maps.a[prob];
+      const CUtensorMap* map_b = &maps.b[prob];
+      const CUtensorMap* map_b32 = &maps.b32[prob];
       const int m0 = (tile / p.n_tiles) * 256 + 128 * (int)rank;
       // this CTA's half of the tile's columns: 128 of a full tile, fewer of a narrow last one.
       // B arrives in boxes of 64 columns (output dimension contiguous) or, for a narrow tile
@@ -627,19 +641,19 @@ mp_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a,
           if (leader) ptx::mbar_arrive_expect_tx(&bars->full[stage], 2 * (HALF_BYTES + b_bytes));
           const int k = kb * BK;
           if (A_MN) {
-            ptx::tma_load_2d_pair(sA, &map_a, full, m0, k);
-            ptx::tma_load_2d_pair(sA + CHUNK_BYTES, &map_a, full, m0 + 64, k);
+            ptx::tma_load_2d_pair(sA, map_a, full, m0, k);
+            ptx::tma_load_2d_pair(sA + CHUNK_BYTES, map_a, full, m0 + 64, k);
           } else {
-            ptx::tma_load_2d_pair(sA, &map_a, full, k, m0);
+            ptx::tma_load_2d_pair(sA, map_a, full, k, m0);
           }
           if (B_MN) {
-            ptx::tma_load_2d_pair(sB, &map_b, full, n0, k);
-            if (b_boxes > 1) ptx::tma_load_2d_pair(sB + CHUNK_BYTES, &map_b, full, n0 + 64, k);
+            ptx::tma_load_2d_pair(sB, map_b, full, n0, k);
+            if (b_boxes > 1) ptx::tma_load_2d_pair(sB + CHUNK_BYTES, map_b, full, n0 + 64, k);
           } else if (b_boxes == 4) {
-            ptx::tma_load_2d_pair(sB, &map_b, full, k, n0);
+            ptx::tma_load_2d_pair(sB, map_b, full, k, n0);
           } else {
             for (int c = 0; c < b_boxes; ++c)   // 32 rows of 128 B each: 4 KiB apart, whole swizzle groups
-              ptx::tma_load_2d_pair(sB + c * (32 * BK * 2), &map_b32, full, k, n0 + 32 * c);
+              ptx::tma_load_2d_pair(sB + c * (32 * BK * 2), map_b32, full, k, n0 + 32 * c);
           }
         }
         __syncwarp();
@@ -666,7 +680,8 @@ mp_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a,
       int iter = 0;
       bool ok = true;
       for (int w = pair; w < total_work && ok; w += npairs, ++iter) {
-        const int split = w % p.splits, tile = w / p.splits;
+        const int wl = w % p.work_per_problem;
+        const int split = wl % p.splits, tile = wl / p.splits;
         const uint32_t idesc =
             ptx::idesc_f16_f32(256, tile_width(p.No, (tile % p.n_tiles) * BN), A_MN, B_MN);
         const int kb0 = (int)((int64_t)split * p.num_kb / p.splits);
@@ -711,7 +726,8 @@ mp_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a,
     int iter = 0;
     bool ok = true;
     for (int w = pair; w < total_work && ok; w += npairs, ++iter) {
-      const int split = w % p.splits, tile = w / p.splits;
+      const int prob = w / p.work_per_problem, wl = w - prob * p.work_per_problem;
+      const int split = wl % p.splits, tile = wl / p.splits;
       const int m0 = (tile / p.n_tiles) * 256 + 128 * (int)rank, n0 = (tile % p.n_tiles) * BN;
       const int acc = iter & 1;
       const uint32_t acc_phase = (iter >> 1) & 1;
@@ -722,9 +738,9 @@ mp_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a,
       if (!ptx::mbar_wait(&bars->tmem_full[acc], acc_phase)) { ok = false; break; }
       ptx::tc_fence_after_sync();
       const uint32_t bad =
-          epilogue_tile<WIDE>(p, &map_out, &map_ws, stage, nslots, stores,
+          epilogue_tile<WIDE>(p, &maps.out[prob], &maps.ws[prob], stage, nslots, stores,
                         tmem_base + acc * BN + ((uint32_t)(q * 32) << 16), row, n0, split, c_begin,
-                        c_count, masked ? pass_bits : nullptr);
+                        c_count, prob, masked ? pass_bits : nullptr);
       if (p.out_mode == OUT_F16_FLAG && p.flag != nullptr) {
         if (__any_sync(0xFFFFFFFFu, bad != 0) && lane == 0) atomicOr(p.flag, 1);
       }
@@ -853,11 +869,11 @@ int make_map_ws(CUtensorMap* map, const void* ptr, int64_t ld, int64_t rows, int
 // Output tiles of more than 128 rows go to the CTA-pair kernel (256 x 256 tiles, one per SM pair).
 bool use_pair_kernel(int64_t Mo) { return Mo > 128; }
 
-int choose_splits(int64_t Mo, int64_t No, int64_t R) {
+int choose_splits(int64_t Mo, int64_t No, int64_t R, int64_t count = 1) {
   const bool pair = use_pair_kernel(Mo);
   const int64_t bm = pair ? 256 : BM;
   const int64_t slots = pair ? kModelSMs / 2 : kModelSMs;
-  const int64_t tiles = ((Mo + bm - 1) / bm) * ((No + BN - 1) / BN);
+  const int64_t tiles = count * ((Mo + bm - 1) / bm) * ((No + BN - 1) / BN);
   const int64_t num_kb = (R + BK - 1) / BK;
   const double t_kb = 0.42e-6;                   // one 128x256x64 block per SM at ~1.0e13 flop/s
   const double bw = 4.0e12;                      // workspace traffic, bytes/s
@@ -867,7 +883,7 @@ int choose_splits(int64_t Mo, int64_t No, int64_t R) {
     const int64_t work = tiles * s;
     const int64_t waves = (work + slots - 1) / slots;
     double t = (double)waves * (double)((num_kb + s - 1) / s) * t_kb;
-    if (s > 1) t += (double)Mo * (double)No * (8.0 * s + 2.0) / bw + 3e-6;
+    if (s > 1) t += (double)count * ((double)Mo * (double)No * (8.0 * s + 2.0) / bw + 3e-6);
     if (t < best_t * 0.97) { best_t = t; best = s; }
   }
   return best;
@@ -891,8 +907,7 @@ struct Operand {
 };
 
 template <bool A_MN, bool B_MN, bool WIDE>
-int launch(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mo, const CUtensorMap& mw,
-           const GemmParams& p, int grid, cudaStream_t st) {
+int launch(const GroupMaps& maps, const GemmParams& p, int grid, cudaStream_t st) {
   static bool attr_set = false;
   if (!attr_set) {
     MP_CUDA_TRY(cudaFuncSetAttribute(mp_gemm_kernel<A_MN, B_MN, WIDE>,
@@ -909,15 +924,13 @@ int launch(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mo, 
   attr.val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = &attr;
   cfg.numAttrs = 1;
-  MP_CUDA_TRY(cudaLaunchKernelEx(&cfg, mp_gemm_kernel<A_MN, B_MN, WIDE>, ma, mb, mo, mw, p));
+  MP_CUDA_TRY(cudaLaunchKernelEx(&cfg, mp_gemm_kernel<A_MN, B_MN, WIDE>, maps, p));
   mp::count_launch();
   return MP_OK;
 }
 
 template <bool A_MN, bool B_MN, bool WIDE>
-int launch_pair(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mb32,
-                const CUtensorMap& mo, const CUtensorMap& mw, const GemmParams& p, int64_t work,
-                cudaStream_t st) {
+int launch_pair(const GroupMaps& maps, const GemmParams& p, int64_t work, cudaStream_t st) {
   static int max_pairs = 0;
   if (max_pairs == 0) {
     MP_CUDA_TRY(cudaFuncSetAttribute(mp_gemm_pair_kernel<A_MN, B_MN, WIDE>,
@@ -947,16 +960,22 @@ int launch_pair(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap&
   attr.val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = &attr;
   cfg.numAttrs = 1;
-  MP_CUDA_TRY(cudaLaunchKernelEx(&cfg, mp_gemm_pair_kernel<A_MN, B_MN, WIDE>, ma, mb, mb32, mo, mw, p));
+  MP_CUDA_TRY(cudaLaunchKernelEx(&cfg, mp_gemm_pair_kernel<A_MN, B_MN, WIDE>, maps, p));
   mp::count_launch();
   return MP_OK;
 }
 
-int run_gemm(const char* name, const Operand& A, const Operand& B, void* out, int64_t ldo,
-             int* flag, bool want_flag, void* workspace, size_t ws_bytes, cudaStream_t st,
+// `count` products of one shape and one set of layouts (operands As[i], Bs[i], outputs outs[i]).
+int run_gemm(const char* name, int count, const Operand* As, const Operand* Bs, void* const* outs,
+             int64_t ldo, int* flag, bool want_flag, void* workspace, size_t ws_bytes, cudaStream_t st,
              const Fuse& fuse = Fuse()) {
+  if (count < 1 || count > MAX_GROUP)
+    return mp::set_error(MP_ERR_INVALID_ARG, "%s: between 1 and %d problems per call", name, MAX_GROUP);
+  const Operand& A = As[0];
+  const Operand& B = Bs[0];
   const int64_t Mo = A.mn, No = B.mn, R = A.red;
-  if (!A.ptr || !B.ptr || !out) return mp::set_error(MP_ERR_INVALID_ARG, "%s: null pointer", name);
+  for (int i = 0; i < count; ++i)
+    if (!As[i].ptr || !Bs[i].ptr || !outs[i]) return mp::set_error(MP_ERR_INVALID_ARG, "%s: null pointer", name);
   if (Mo <= 0 || No <= 0 || R <= 0)
     return mp::set_error(MP_ERR_INVALID_ARG, "%s: sizes must be positive", name);
   if (Mo > INT32_MAX / 2 || No > INT32_MAX / 2 || R > INT32_MAX / 2)
@@ -966,60 +985,74 @@ int run_gemm(const char* name, const Operand& A, const Operand& B, void* out, in
     return mp::set_error(MP_ERR_INVALID_ARG, "%s: leading dimension smaller than the row length", name);
   if ((A.ld | B.ld | ldo) & 7)
     return mp::set_error(MP_ERR_ALIGNMENT, "%s: leading dimensions must be multiples of 8", name);
-  if (!mp::aligned16(A.ptr) || !mp::aligned16(B.ptr) || !mp::aligned16(out) ||
-      (workspace && !mp::aligned16(workspace)))
+  for (int i = 0; i < count; ++i)
+    if (!mp::aligned16(As[i].ptr) || !mp::aligned16(Bs[i].ptr) || !mp::aligned16(outs[i]))
+      return mp::set_error(MP_ERR_ALIGNMENT, "%s: pointers must be 16-byte aligned", name);
+  if (workspace && !mp::aligned16(workspace))
     return mp::set_error(MP_ERR_ALIGNMENT, "%s: pointers must be 16-byte aligned", name);
   if (int rc = mp::check_device()) return rc;
   if (int rc = load_encoder()) return rc;
 
   const int64_t No8 = No & ~(int64_t)7;
   GemmParams p;
+  p.group = count;
   p.Mo = (int)Mo; p.No = (int)No; p.R = (int)R; p.No8 = (int)No8;
   const bool pair = use_pair_kernel(Mo);
   p.m_tiles = (int)(pair ? (Mo + 255) / 256 : (Mo + BM - 1) / BM);
   p.n_tiles = (int)((No + BN - 1) / BN);
   p.num_kb = (int)((R + BK - 1) / BK);
   const bool fused = fuse.bias != nullptr || fuse.act != 0;
-  p.splits = fused ? 1 : choose_splits(Mo, No, R);   // the fused epilogue needs the whole sum
+  if (fused && count != 1)
+    return mp::set_error(MP_ERR_INVALID_ARG, "%s: the fused epilogues take one problem per call", name);
+  p.splits = fused ? 1 : choose_splits(Mo, No, R, count);   // the fused epilogue needs the whole sum
+  p.work_per_problem = p.m_tiles * p.n_tiles * p.splits;
   p.bias = (const uint16_t*)fuse.bias; p.mask = (const uint16_t*)fuse.mask;
   p.ldmask = fuse.ldmask; p.act = fuse.act; p.clip = fuse.clip;
-  p.out = (uint16_t*)out; p.ldo = ldo;
+  for (int i = 0; i < MAX_GROUP; ++i) p.out[i] = (uint16_t*)outs[i < count ? i : 0];
+  p.ldo = ldo;
   p.ws = (float*)workspace; p.ws_ld = ws_ld_for(No);
   p.flag = flag;
   p.out_mode = p.splits > 1 ? OUT_PARTIAL : (want_flag ? OUT_F16_FLAG : OUT_F16);
+  const size_t ws_floats_per_problem = (size_t)p.splits * (size_t)Mo * (size_t)p.ws_ld;
   if (p.splits > 1) {
-    const size_t need = (size_t)p.splits * (size_t)Mo * (size_t)p.ws_ld * sizeof(float);
+    const size_t need = (size_t)count * ws_floats_per_problem * sizeof(float);
     if (!workspace || ws_bytes < need)
       return mp::set_error(MP_ERR_NOMEM, "%s: workspace of %zu bytes needed, %zu given", name, need,
                            workspace ? ws_bytes : (size_t)0);
   }
 
-  CUtensorMap ma, mb, mb32, mo, mw;
-  // FP16 output: 32-row x 64-column boxes, the unit one epilogue warp stores at a time
-  // (first No8 columns; a map over 8 columns that is never used when No < 8)
-  if (int rc = make_map(&mo, out, No8 > 0 ? No8 : 8, Mo, ldo, 64, 32)) return rc;
-  if (int rc = A.mn_major ? make_map(&ma, A.ptr, A.mn, A.red, A.ld, 64, BK)
-                          : make_map(&ma, A.ptr, A.red, A.mn, A.ld, BK, BM)) return rc;
-  if (int rc = B.mn_major ? make_map(&mb, B.ptr, B.mn, B.red, B.ld, 64, BK)
-                          : make_map(&mb, B.ptr, B.red, B.mn, B.ld, BK, pair ? 128 : BN)) return rc;
-  // reduction-contiguous B of the pair kernel: 32-row boxes for a narrow last column tile
-  if (pair && !B.mn_major) {
-    if (int rc = make_map(&mb32, B.ptr, B.red, B.mn, B.ld, BK, 32)) return rc;
-  } else {
-    mb32 = mb;
+  GroupMaps maps;
+  for (int i = 0; i < count; ++i) {
+    // FP16 output: 32-row x 64-column boxes, the unit one epilogue warp stores at a time
+    // (first No8 columns; a map over 8 columns that is never used when No < 8)
+    if (int rc = make_map(&maps.out[i], outs[i], No8 > 0 ? No8 : 8, Mo, ldo, 64, 32)) return rc;
+    if (int rc = A.mn_major ? make_map(&maps.a[i], As[i].ptr, A.mn, A.red, A.ld, 64, BK)
+                            : make_map(&maps.a[i], As[i].ptr, A.red, A.mn, A.ld, BK, BM)) return rc;
+    if (int rc = B.mn_major ? make_map(&maps.b[i], Bs[i].ptr, B.mn, B.red, B.ld, 64, BK)
+                            : make_map(&maps.b[i], Bs[i].ptr, B.red, B.mn, B.ld, BK, pair ? 128 : BN)) return rc;
+    // reduction-contiguous B of the pair kernel: 32-row boxes for a narrow last column tile
+    if (pair && !B.mn_major) {
+      if (int rc = make_map(&maps.b32[i], Bs[i].ptr, B.red, B.mn, B.ld, BK, 32)) return rc;
+    } else {
+      maps.b32[i] = maps.b[i];
+    }
+    // FP32 partial sums of a split reduction: [split][row][padded column], boxes of 32 x 32 floats
+    if (p.splits > 1) {
+      if (int rc = make_map_ws(&maps.ws[i], p.ws + (size_t)i * ws_floats_per_problem, p.ws_ld, Mo, p.splits))
+        return rc;
+    } else {
+      maps.ws[i] = maps.out[i];
+    }
   }
-
-  // FP32 partial sums of a split reduction: [split][row][padded column], boxes of 32 x 32 floats
-  if (p.splits > 1) {
-    if (int rc = make_map_ws(&mw, workspace, p.ws_ld, Mo, p.splits)) return rc;
-  } else {
-    mw = mo;
+  for (int i = count; i < MAX_GROUP; ++i) {       // unused entries: valid copies of problem 0
+    maps.a[i] = maps.a[0]; maps.b[i] = maps.b[0]; maps.b32[i] = maps.b32[0];
+    maps.out[i] = maps.out[0]; maps.ws[i] = maps.ws[0];
   }
 
   int dev = 0, sms = 0;
   MP_CUDA_TRY(cudaGetDevice(&dev));
   MP_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-  const int64_t work = (int64_t)p.m_tiles * p.n_tiles * p.splits;
+  const int64_t work = (int64_t)count * p.work_per_problem;
   const int grid = (int)(work < sms ? work : sms);
 
   // eight epilogue warps (two per scheduler) for the bias / activation / mask flavours, four for
@@ -1032,8 +1065,8 @@ int run_gemm(const char* name, const Operand& A, const Operand& B, void* out, in
     else if (!A.mn_major && !B.mn_major) rc = fused ? FN<false, false, true>(__VA_ARGS__) : FN<false, false, false>(__VA_ARGS__); \
     else rc = fused ? FN<true, false, true>(__VA_ARGS__) : FN<true, false, false>(__VA_ARGS__); \
   } while (0)
-  if (pair) MP_DISPATCH(launch_pair, ma, mb, mb32, mo, mw, p, work, st);
-  else MP_DISPATCH(launch, ma, mb, mo, mw, p, grid, st);
+  if (pair) MP_DISPATCH(launch_pair, maps, p, work, st);
+  else MP_DISPATCH(launch, maps, p, grid, st);
 #undef MP_DISPATCH
   if (rc) return rc;
 
@@ -1041,35 +1074,93 @@ int run_gemm(const char* name, const Operand& A, const Operand& B, void* out, in
     const int64_t vecs = Mo * ((No + 3) / 4);
     int64_t blocks = (vecs + 255) / 256;
     if (blocks > (int64_t)sms * 8) blocks = (int64_t)sms * 8;
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)blocks, 1, 1);
-    cfg.blockDim = dim3(256, 1, 1);
-    cfg.stream = st;
-    cudaLaunchAttribute attr;
-    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr.val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = &attr;
-    cfg.numAttrs = 1;
-    MP_CUDA_TRY(cudaLaunchKernelEx(&cfg, mp_splitk_reduce_kernel, (const float*)p.ws, p.splits, p.Mo,
-                                   p.No, p.ws_ld, p.out, p.ldo, want_flag ? flag : (int*)nullptr));
-    mp::count_launch();
+    for (int i = 0; i < count; ++i) {
+      cudaLaunchConfig_t cfg = {};
+      cfg.gridDim = dim3((unsigned)blocks, 1, 1);
+      cfg.blockDim = dim3(256, 1, 1);
+      cfg.stream = st;
+      cudaLaunchAttribute attr;
+      attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+      attr.val.programmaticStreamSerializationAllowed = 1;
+      cfg.attrs = &attr;
+      cfg.numAttrs = 1;
+      MP_CUDA_TRY(cudaLaunchKernelEx(&cfg, mp_splitk_reduce_kernel,
+                                     (const float*)(p.ws + (size_t)i * ws_floats_per_problem), p.splits, p.Mo,
+                                     p.No, p.ws_ld, p.out[i], p.ldo, want_flag ? flag : (int*)nullptr));
+      mp::count_launch();
+    }
   }
   return MP_OK;
+}
+
+// One product: the common case.
+int run_gemm(const char* name, const Operand& A, const Operand& B, void* out, int64_t ldo, int* flag,
+             bool want_flag, void* workspace, size_t ws_bytes, cudaStream_t st, const Fuse& fuse = Fuse()) {
+  void* outs[1] = {out};
+  return run_gemm(name, 1, &A, &B, outs, ldo, flag, want_flag, workspace, ws_bytes, st, fuse);
+}
+
+// Output rows, output columns and reduction length of a layer's product `op`.
+bool product_dims(int64_t M, int64_t K, int64_t N, int op, int64_t* Mo, int64_t* No, int64_t* R) {
+  if (op == MP_OP_FWD) { *Mo = M; *No = N; *R = K; }
+  else if (op == MP_OP_DGRAD) { *Mo = M; *No = K; *R = N; }
+  else if (op == MP_OP_WGRAD) { *Mo = K; *No = N; *R = M; }
+  else return false;
+  return true;
 }
 
 }  // namespace
 
 extern "C" {
 
-size_t mp_gemm_workspace_bytes(int64_t M, int64_t K, int64_t N, int op) {
-  if (M <= 0 || K <= 0 || N <= 0) return 0;
+size_t mp_gemm_workspace_bytes_grouped(int count, int64_t M, int64_t K, int64_t N, int op) {
+  if (M <= 0 || K <= 0 || N <= 0 || count < 1 || count > MAX_GROUP) return 0;
   int64_t Mo, No, R;
-  if (op == MP_OP_FWD) { Mo = M; No = N; R = K; }
-  else if (op == MP_OP_DGRAD) { Mo = M; No = K; R = N; }
-  else if (op == MP_OP_WGRAD) { Mo = K; No = N; R = M; }
-  else return 0;
-  const int s = choose_splits(Mo, No, R);
-  return s > 1 ? (size_t)s * (size_t)Mo * (size_t)ws_ld_for(No) * sizeof(float) : 0;
+  if (!product_dims(M, K, N, op, &Mo, &No, &R)) return 0;
+  const int s = choose_splits(Mo, No, R, count);
+  return s > 1 ? (size_t)count * (size_t)s * (size_t)Mo * (size_t)ws_ld_for(No) * sizeof(float) : 0;
+}
+
+size_t mp_gemm_workspace_bytes(int64_t M, int64_t K, int64_t N, int op) {
+  return mp_gemm_workspace_bytes_grouped(1, M, K, N, op);
+}
+
+int mp_max_group(void) { return MAX_GROUP; }
+
+// ---- several independent layers of one shape in one launch ---------------------------------
+int mp_linear_fwd_grouped(int count, const void* const* X16, int64_t ldx, const void* const* W16,
+                          int64_t ldw, void* const* Y16, int64_t ldy, int64_t M, int64_t K, int64_t N,
+                          void* workspace, size_t workspace_bytes, void* stream) {
+  if (count < 1 || count > MAX_GROUP || !X16 || !W16 || !Y16)
+    return mp::set_error(MP_ERR_INVALID_ARG, "mp_linear_fwd_grouped: 1..%d problems, non-null arrays", MAX_GROUP);
+  Operand A[MAX_GROUP], B[MAX_GROUP];
+  for (int i = 0; i < count; ++i) { A[i] = Operand{X16[i], ldx, false, M, K}; B[i] = Operand{W16[i], ldw, true, N, K}; }
+  return run_gemm("mp_linear_fwd_grouped", count, A, B, Y16, ldy, nullptr, false, workspace, workspace_bytes,
+                  (cudaStream_t)stream);
+}
+
+int mp_linear_bwd_dgrad_grouped(int count, const void* const* dY16, int64_t lddy, const void* const* W16,
+                                int64_t ldw, void* const* dX16, int64_t lddx, int64_t M, int64_t K,
+                                int64_t N, void* workspace, size_t workspace_bytes, void* stream) {
+  if (count < 1 || count > MAX_GROUP || !dY16 || !W16 || !dX16)
+    return mp::set_error(MP_ERR_INVALID_ARG, "mp_linear_bwd_dgrad_grouped: 1..%d problems, non-null arrays", MAX_GROUP);
+  Operand A[MAX_GROUP], B[MAX_GROUP];
+  for (int i = 0; i < count; ++i) { A[i] = Operand{dY16[i], lddy, false, M, N}; B[i] = Operand{W16[i], ldw, false, K, N}; }
+  return run_gemm("mp_linear_bwd_dgrad_grouped", count, A, B, dX16, lddx, nullptr, false, workspace,
+                  workspace_bytes, (cudaStream_t)stream);
+}
+
+int mp_linear_bwd_wgrad_grouped(int count, const void* const* X16, int64_t ldx, const void* const* dY16,
+                                int64_t lddy, void* const* dW16, int64_t lddw, int64_t M, int64_t K,
+                                int64_t N, mp_state* state, void* workspace, size_t workspace_bytes,
+                                void* stream) {
+  if (count < 1 || count > MAX_GROUP || !X16 || !dY16 || !dW16)
+    return mp::set_error(MP_ERR_INVALID_ARG, "mp_linear_bwd_wgrad_grouped: 1..%d problems, non-null arrays", MAX_GROUP);
+  Operand A[MAX_GROUP], B[MAX_GROUP];
+  for (int i = 0; i < count; ++i) { A[i] = Operand{X16[i], ldx, true, K, M}; B[i] = Operand{dY16[i], lddy, true, N, M}; }
+  int* flag = state ? &state->dev->h.found_inf : nullptr;
+  return run_gemm("mp_linear_bwd_wgrad_grouped", count, A, B, dW16, lddw, flag, state != nullptr, workspace,
+                  workspace_bytes, (cudaStream_t)stream);
 }
 
 int mp_linear_fwd(const void* X16, int64_t ldx, const void* W16, int64_t ldw, void* Y16,

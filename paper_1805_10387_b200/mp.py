@@ -61,6 +61,11 @@ SIGNATURES = {
     "mp_linear_bwd_wgrad": (_i32, [_p, _i64, _p, _i64, _p, _i64, _i64, _i64, _i64, _p, _p, _sz, _p]),
     "mp_linear_bwd_wgrad_static": (_i32, [_p, _i64, _p, _i64, _p, _i64, _i64, _i64, _i64, _p, _p]),
     "mp_static_scratch_bytes": (_sz, []),
+    "mp_linear_fwd_grouped": (_i32, [_i32, _p, _i64, _p, _i64, _p, _i64, _i64, _i64, _i64, _p, _sz, _p]),
+    "mp_linear_bwd_dgrad_grouped": (_i32, [_i32, _p, _i64, _p, _i64, _p, _i64, _i64, _i64, _i64, _p, _sz, _p]),
+    "mp_linear_bwd_wgrad_grouped": (_i32, [_i32, _p, _i64, _p, _i64, _p, _i64, _i64, _i64, _i64, _p, _p, _sz, _p]),
+    "mp_max_group": (_i32, []),
+    "mp_gemm_workspace_bytes_grouped": (_sz, [_i32, _i64, _i64, _i64, _i32]),
     "mp_linear_fwd_act": (_i32, [_p, _i64, _p, _i64, _p, _p, _i64, _i64, _i64, _i64, _i32, C.c_float, _p, _sz, _p]),
     "mp_linear_bwd_dgrad_act": (_i32, [_p, _i64, _p, _i64, _p, _i64, _p, _i64, _i64, _i64, _i64, _i32,
                                        C.c_float, _p, _sz, _p]),
@@ -185,6 +190,44 @@ def mp_linear_bwd_wgrad_static(X16, dY16, dW16, state=None):
     assert dY16.shape[0] == M and tuple(dW16.shape) == (K, N)
     _check(lib().mp_linear_bwd_wgrad_static(x, ldx, dy, lddy, dw, lddw, M, K, N,
                                             state.handle if state is not None else None, _stream()))
+
+
+def mp_max_group() -> int:
+    return int(lib().mp_max_group())
+
+
+def mp_gemm_workspace_bytes_grouped(count: int, M: int, K: int, N: int, op: int) -> int:
+    return int(lib().mp_gemm_workspace_bytes_grouped(count, M, K, N, op))
+
+
+def _mats(ts):
+    """(array of pointers, common leading dimension, common shape) of same-shaped 2-D FP16 tensors."""
+    pl = [_mat(t) for t in ts]
+    assert len({ld for _, ld in pl}) == 1 and len({tuple(t.shape) for t in ts}) == 1, \
+        "grouped problems share one shape and one leading dimension"
+    return (C.c_void_p * len(ts))(*[p for p, _ in pl]), pl[0][1], tuple(ts[0].shape)
+
+
+def mp_linear_fwd_grouped(X16s, W16s, Y16s, workspace=None):
+    (x, ldx, (M, K)), (w, ldw, (K2, N)), (y, ldy, ys) = _mats(X16s), _mats(W16s), _mats(Y16s)
+    assert K2 == K and ys == (M, N) and len(X16s) == len(W16s) == len(Y16s)
+    ws, nb = _ws(workspace)
+    _check(lib().mp_linear_fwd_grouped(len(X16s), x, ldx, w, ldw, y, ldy, M, K, N, ws, nb, _stream()))
+
+
+def mp_linear_bwd_dgrad_grouped(dY16s, W16s, dX16s, workspace=None):
+    (dy, lddy, (M, N)), (w, ldw, (K, N2)), (dx, lddx, xs) = _mats(dY16s), _mats(W16s), _mats(dX16s)
+    assert N2 == N and xs == (M, K) and len(dY16s) == len(W16s) == len(dX16s)
+    ws, nb = _ws(workspace)
+    _check(lib().mp_linear_bwd_dgrad_grouped(len(dY16s), dy, lddy, w, ldw, dx, lddx, M, K, N, ws, nb, _stream()))
+
+
+def mp_linear_bwd_wgrad_grouped(X16s, dY16s, dW16s, state=None, workspace=None):
+    (x, ldx, (M, K)), (dy, lddy, (M2, N)), (dw, lddw, ws_) = _mats(X16s), _mats(dY16s), _mats(dW16s)
+    assert M2 == M and ws_ == (K, N) and len(X16s) == len(dY16s) == len(dW16s)
+    ws, nb = _ws(workspace)
+    _check(lib().mp_linear_bwd_wgrad_grouped(len(X16s), x, ldx, dy, lddy, dw, lddw, M, K, N,
+                                             state.handle if state is not None else None, ws, nb, _stream()))
 
 
 def mp_static_scratch_bytes() -> int:

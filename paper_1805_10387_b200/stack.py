@@ -103,7 +103,26 @@ class LinearStack:
                 self.dy[l] = self.dy_top_flat[flat_off[l]:flat_off[l] + m * n].view(m, n)
             else:
                 self.dy[l] = torch.zeros(self.shapes[l][0], _align(self.shapes[l][2]), **f16)
+        # Runs of consecutive layers that depend on nothing in the stack (no chained input, output
+        # feeding no layer), have one shape and plain epilogues go to the grouped calls, a few
+        # layers per launch; every other layer is a group of one.
+        self.groups = []
+        gmax = mp.mp_max_group()
+        for l in range(self.L):
+            free = (not self.chained[l] and not (l + 1 < self.L and self.chained[l + 1])
+                    and self.acts[l] == mp.MP_ACT_NONE and not self.has_bias)
+            g = self.groups[-1] if self.groups else None
+            if (free and g is not None and g[1] and len(g[0]) < gmax
+                    and self.shapes[g[0][0]] == self.shapes[l]):
+                g[0].append(l)
+            else:
+                self.groups.append(([l], free))
+        self.groups = [g[0] for g in self.groups]
         need = 0
+        for g in self.groups:
+            m, k, n = self.shapes[g[0]]
+            for op in (mp.MP_OP_FWD, mp.MP_OP_DGRAD, mp.MP_OP_WGRAD):
+                need = max(need, mp.mp_gemm_workspace_bytes_grouped(len(g), m, k, n, op))
         for m, k, n in self.shapes:
             for op in (mp.MP_OP_FWD, mp.MP_OP_DGRAD, mp.MP_OP_WGRAD):
                 need = max(need, mp.mp_gemm_workspace_bytes(m, k, n, op))
@@ -272,37 +291,52 @@ class LinearStack:
         for l in range(self.L):
             if not self.chained[l]:
                 self.x[l] = xs[l]
-            if self.acts[l] == mp.MP_ACT_NONE and not self.has_bias:
-                self._call("fwd", mp.mp_linear_fwd, self.x[l][:, :self.shapes[l][1]], self.W16(l), self.Y(l),
-                           self.workspace)
-            else:
-                self._call("fwd", mp.mp_linear_fwd_act, self.x[l][:, :self.shapes[l][1]], self.W16(l),
-                           self.b16[l], self.Y(l), self.acts[l], self.clip, self.workspace)
+        Xv = lambda l: self.x[l][:, :self.shapes[l][1]]
+        for g in self.groups:
+            if len(g) > 1 and len({self.x[l].stride(0) for l in g}) == 1:
+                self._call("fwd", mp.mp_linear_fwd_grouped, [Xv(l) for l in g], [self.W16(l) for l in g],
+                           [self.Y(l) for l in g], self.workspace)
+                continue
+            for l in g:
+                if self.acts[l] == mp.MP_ACT_NONE and not self.has_bias:
+                    self._call("fwd", mp.mp_linear_fwd, Xv(l), self.W16(l), self.Y(l), self.workspace)
+                else:
+                    self._call("fwd", mp.mp_linear_fwd_act, Xv(l), self.W16(l), self.b16[l], self.Y(l),
+                               self.acts[l], self.clip, self.workspace)
         g_flat = self._flat_upstream(gs)
         if g_flat is not None:        # one scaling call for all flat top layers
             self._call("scale", mp.mp_scale_upstream, g_flat, self.dy_top_flat, self.state)
-        for l in range(self.L - 1, -1, -1):
-            if not self.feeds_next(l) and not (g_flat is not None and l in self.flat_tops):
-                n = self.shapes[l][2]
-                if self.dy[l].shape[1] == n:
-                    self._call("scale", mp.mp_scale_upstream, gs[l], self.dy[l], self.state)
-                elif self.only is None or "scale" in self.only:
-                    # padded rows: scale into a dense buffer, then place (copy only)
-                    tmp = torch.empty(self.shapes[l][0], n, dtype=torch.float16, device=self.device)
-                    mp.mp_scale_upstream(gs[l], tmp, self.state)
-                    self.dy[l][:, :n].copy_(tmp)
-            X = self.x[l][:, :self.shapes[l][1]]
-            self._call("wgrad", mp.mp_linear_bwd_wgrad, X, self.dY(l), self.dW(l), self.state,
-                       self.workspace)
-            if self.has_bias:
-                self._call("bgrad", mp.mp_bias_grad, self.dY(l), self.db[l], self.state, self.workspace)
-            below = self.acts[l - 1] if self.chained[l] else mp.MP_ACT_NONE
-            if below == mp.MP_ACT_NONE:
-                self._call("dgrad", mp.mp_linear_bwd_dgrad, self.dY(l), self.W16(l), self.dX(l),
+        for g in reversed(self.groups):
+            for l in reversed(g):
+                if not self.feeds_next(l) and not (g_flat is not None and l in self.flat_tops):
+                    n = self.shapes[l][2]
+                    if self.dy[l].shape[1] == n:
+                        self._call("scale", mp.mp_scale_upstream, gs[l], self.dy[l], self.state)
+                    elif self.only is None or "scale" in self.only:
+                        # padded rows: scale into a dense buffer, then place (copy only)
+                        tmp = torch.empty(self.shapes[l][0], n, dtype=torch.float16, device=self.device)
+                        mp.mp_scale_upstream(gs[l], tmp, self.state)
+                        self.dy[l][:, :n].copy_(tmp)
+            if (len(g) > 1 and len({self.x[l].stride(0) for l in g}) == 1
+                    and len({self.dy[l].stride(0) for l in g}) == 1):
+                self._call("wgrad", mp.mp_linear_bwd_wgrad_grouped, [Xv(l) for l in g], [self.dY(l) for l in g],
+                           [self.dW(l) for l in g], self.state, self.workspace)
+                self._call("dgrad", mp.mp_linear_bwd_dgrad_grouped, [self.dY(l) for l in g],
+                           [self.W16(l) for l in g], [self.dX(l) for l in g], self.workspace)
+                continue
+            for l in reversed(g):
+                X = Xv(l)
+                self._call("wgrad", mp.mp_linear_bwd_wgrad, X, self.dY(l), self.dW(l), self.state,
                            self.workspace)
-            else:       # the layer below is activated: mask with its stored output (= this layer's input)
-                self._call("dgrad", mp.mp_linear_bwd_dgrad_act, self.dY(l), self.W16(l), X, self.dX(l),
-                           below, self.clip, self.workspace)
+                if self.has_bias:
+                    self._call("bgrad", mp.mp_bias_grad, self.dY(l), self.db[l], self.state, self.workspace)
+                below = self.acts[l - 1] if self.chained[l] else mp.MP_ACT_NONE
+                if below == mp.MP_ACT_NONE:
+                    self._call("dgrad", mp.mp_linear_bwd_dgrad, self.dY(l), self.W16(l), self.dX(l),
+                               self.workspace)
+                else:   # the layer below is activated: mask with its stored output (= this layer's input)
+                    self._call("dgrad", mp.mp_linear_bwd_dgrad_act, self.dY(l), self.W16(l), X, self.dX(l),
+                               below, self.clip, self.workspace)
         if self.grad_sync is not None and self.only is None:   # data parallel: sum the FP16 gradients over ranks,
             self.grad_sync(self.dw_flat)     # then inspect the reduced gradients in the update call
         self._call("update", mp.mp_master_update, self.plan, self.state, self.opt,

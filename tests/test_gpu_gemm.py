@@ -118,6 +118,52 @@ def test_every_width_of_the_last_column_tile(orc, mp, op, width):
         assert got.shape == want.shape and (got == want).all(), (op, rows, width)
 
 
+@pytest.mark.parametrize("op", ["fwd", "dgrad", "wgrad"])
+@pytest.mark.parametrize("M,K,N,count", [(300, 200, 264, 3), (70, 136, 40, 4), (4096, 128, 256, 2),
+                                         (1024, 512, 512, 4), (520, 72, 29, 2)])
+def test_grouped_call_equals_single_calls(orc, mp, op, M, K, N, count):
+    """Several independent products of one shape in one launch: with integer operands (sums exact
+    in any order, so a different reduction split cannot show) every problem's output is bit for
+    bit the oracle's and the single call's; nothing is written outside any output."""
+    rng = np.random.default_rng(M + K + N + count)
+    sa, sb = _shapes_for(op, M, K, N)
+    As = [_h(rng.integers(-2, 3, sa)) for _ in range(count)]
+    Bs = [_h(rng.integers(-2, 3, sb)) for _ in range(count)]
+    oshape = {"fwd": (M, N), "dgrad": (M, K), "wgrad": (K, N)}[op]
+    outs = [_out(*oshape) for _ in range(count)]
+    opi = {"fwd": 0, "dgrad": 1, "wgrad": 2}[op]
+    ws = torch.empty(max(mp.mp_gemm_workspace_bytes_grouped(count, M, K, N, opi), 16), dtype=torch.uint8, device="cuda")
+    ws.fill_(0x7F)                                      # stale scratch must not matter
+    dA, dB = [_to_dev(a) for a in As], [_to_dev(b) for b in Bs]
+    st = mp.State()
+    if op == "fwd":
+        mp.mp_linear_fwd_grouped(dA, dB, [o for o, _ in outs], ws)
+    elif op == "dgrad":
+        mp.mp_linear_bwd_dgrad_grouped(dA, dB, [o for o, _ in outs], ws)
+    else:
+        mp.mp_linear_bwd_wgrad_grouped(dA, dB, [o for o, _ in outs], st, ws)
+    torch.cuda.synchronize()
+    assert mp.mp_gemm_device_status() == 0 and st.read().found_inf == 0
+    for i in range(count):
+        out, raw = outs[i]
+        assert bool((raw[:, out.shape[1]:] == 0x5A5A).all())
+        assert bool((raw[:GUARD_ROWS] == 0x5A5A).all()) and bool((raw[-GUARD_ROWS:] == 0x5A5A).all())
+        want = _oracle(orc, op, As[i], Bs[i])
+        assert (_bits(out) == want).all(), (op, i)
+        single, _ = _run(mp, op, As[i], Bs[i])
+        assert (single == want).all()
+    st.close()
+
+
+def test_grouped_call_rejects_bad_counts(mp):
+    a = torch.zeros(16, 16, dtype=torch.float16, device="cuda")
+    n = mp.mp_max_group()
+    assert n >= 2 and mp.mp_gemm_workspace_bytes_grouped(n + 1, 64, 64, 64, mp.MP_OP_FWD) == 0
+    with pytest.raises(mp.MpError) as e:
+        mp.mp_linear_fwd_grouped([a] * (n + 1), [a] * (n + 1), [a.clone() for _ in range(n + 1)])
+    assert e.value.code == mp.MP_ERR_INVALID_ARG
+
+
 @pytest.mark.parametrize("op,M,K,N", [("wgrad", 4096, 128, 256), ("wgrad", 3000, 200, 300),
                                       ("fwd", 2048, 2048, 512), ("dgrad", 1500, 640, 2048)])
 def test_integer_exact_large_and_split(orc, mp, op, M, K, N):
