@@ -33,8 +33,10 @@ METRIC = "MP train step: GEMM TFLOP/s and master-update GB/s, % of B200 peak"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 # DRAM bytes per launch of the GEMM kernel from one ncu capture (dram__bytes_read.sum +
-# dram__bytes_write.sum), keyed by workload, valid only for the kernel source it was taken on.
-NCU_TRAFFIC = {"sha": "c79dcfdfe0b8ac28", "bytes_per_launch": {"c2": 81.5e6}}
+# dram__bytes_write.sum, mean over one step's product launches; on c2 a launch holds four layers'
+# products, 4 x 95.4 MB algorithmic), keyed by workload, valid only for the kernel source it was
+# taken on.
+NCU_TRAFFIC = {"sha": "5287f7d542101890", "bytes_per_launch": {"c2": 402.2e6}}
 
 
 def peaks():
