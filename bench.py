@@ -571,6 +571,8 @@ def main():
                      "frac_of_burst_peak": gemm_tflops / pk["bf16_tflops"],
                      "frac_of_nominal_2250": gemm_tflops / 2250.0,
                      "launches": gemm_launches, "avg_launch_ms": gemm_ms / max(gemm_launches, 1),
+                     "algorithmic_gflop_per_launch": flops_step * args.steps / max(gemm_launches, 1) / 1e9,
+                     "grouping": "independent same-shape layers run up to four per launch",
                      "calls": gemm_calls, "timed_in": gemm_how,
                      "per_op_tflops": per_op},
         "update": {"kernel": "mp_master_update_kernel", "bound": "hbm", "achieved": upd_gbs,
