@@ -23,7 +23,8 @@
 //
 // A long reduction with few output tiles (the weight gradient) can be split across CTAs:
 // each split stores FP32 partial sums to a workspace and a second kernel adds them in a
-// fixed order, rounds to FP16 and inspects.
+// fixed order, rounds to FP16 and inspects.  Up to four independent products of one shape can
+// share a launch (the *_grouped entry points): one persistent work list over all their tiles.
 
 #include <cuda.h>
 #include <cudaTypedefs.h>
@@ -41,10 +42,10 @@ constexpr int B_BYTES = BN * BK * 2;           // 32 KiB
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int CHUNK_BYTES = 64 * BK * 2;       // one 64 x 64 box of an MN-major operand
 // warp 0 producer, warp 1 MMA issuer, then 4 or 8 epilogue warps.  Four (one per TMEM lane quarter)
-// are enough when the epilogue only rounds and stores: it hides behind the next tile's main loop.
-// The bias / activation / mask epilogues are bound by the issue rate of one warp per scheduler,
-// so they are launched with eight (two per lane quarter, each taking half of the tile's columns):
-// 137 against 154 us on the masked 25600x1600x1600 data gradient.
+// for the plain flavours, whose epilogue only rounds and stores (eight were measured and are no
+// faster).  The bias / activation / mask epilogues are bound by the issue rate of one warp per
+// scheduler, so they are launched with eight (two per lane quarter, each taking half of the
+// tile's columns): 137 against 154 us on the masked 25600x1600x1600 data gradient.
 constexpr int THREADS_PLAIN = 64 + 32 * 4;
 constexpr int THREADS_FUSED = 64 + 32 * 8;
 constexpr int TMEM_COLS = 512;
@@ -106,13 +107,6 @@ __device__ __forceinline__ void report_timeout(B* bars) {
   atomicCAS(&g_gemm_status, 0, (int)MP_ERR_TIMEOUT);
 }
 
-// Width of the MMAs of the tile whose first column is n_base: the columns that exist, rounded up
-// to 32, at most BN.  A ragged last column tile (1600 = 6 x 256 + 64) then issues a quarter of
-// the MMA work of a full one instead of multiplying zero-filled columns, and the producer
-// fetches only the B boxes those MMAs read (a full tile's loads, 64 B per clock and SM, take
-// as long as its MMAs, so a narrow tile gets faster only if its loads shrink too).  Multiples
-// of 32 keep every form legal: N % 16 == 0 for both instruction shapes, and each CTA of a pair
-// holds N / 2 (a multiple of 16) columns of B.
 // Row-tile and column-tile index of tile number `tile`.  Consecutive tiles run at the same time
 // on the GPU, so the fast index is that of the smaller operand: its panels stay in L2 while the
 // larger operand streams through once (with the column index fast, a weight gradient of 8 x 16
@@ -124,6 +118,13 @@ __device__ __forceinline__ int tile_n(const GemmParams& p, int tile) {
   return p.m_fast ? tile / p.m_tiles : tile % p.n_tiles;
 }
 
+// Width of the MMAs of the tile whose first column is n_base: the columns that exist, rounded up
+// to 32, at most BN.  A ragged last column tile (1600 = 6 x 256 + 64) then issues a quarter of
+// the MMA work of a full one instead of multiplying zero-filled columns, and the producer
+// fetches only the B boxes those MMAs read (a full tile's loads, 64 B per clock and SM, take
+// as long as its MMAs, so a narrow tile gets faster only if its loads shrink too).  Multiples
+// of 32 keep every form legal: N % 16 == 0 for both instruction shapes, and each CTA of a pair
+// holds N / 2 (a multiple of 16) columns of B.
 __device__ __forceinline__ int tile_width(int No, int n_base) {
   const int left = No - n_base;
   return left >= BN ? BN : ((left + 31) & ~31);
