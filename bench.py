@@ -353,12 +353,16 @@ def main():
     L = len(cfg.shapes)
     chained = [cfg.chained(l) for l in range(L)]
     acts = None
-    if args.real_layers:
+    lstm = None
+    if args.real_layers and cfg.name == "c2":      # the gate products feed LSTM cells (no bias, no activation)
+        lstm = [True] * L
+    elif args.real_layers:
         act = mp.MP_ACT_CLIPPED_RELU if cfg.name == "c4" else mp.MP_ACT_RELU
         acts = [act if (l + 1 < L and chained[l + 1]) else mp.MP_ACT_NONE for l in range(L)]
     stack = LinearStack(cfg.shapes, chained, optimizer=cfg.optimizer, lr=cfg.lr, beta1=cfg.beta1,
                         beta2=cfg.beta2, eps=cfg.eps, momentum=cfg.momentum, init_scale=cfg.init_scale,
-                        growth_interval=cfg.growth_interval, acts=acts, bias=args.real_layers)
+                        growth_interval=cfg.growth_interval, acts=acts, bias=args.real_layers and lstm is None,
+                        lstm=lstm)
     if world > 1:      # data parallel over rows: weights replicated, FP16 weight gradients summed
         from paper_1805_10387_b200 import dp
         stack.grad_sync = dp.allreduce_gradients
@@ -366,7 +370,7 @@ def main():
     gen.manual_seed(1234 + cfg.seed)           # same weights on every rank
     for l, (M, K, N) in enumerate(cfg.shapes):
         w = torch.randn(K, N, generator=gen, device="cuda") / K ** 0.5
-        if args.real_layers:
+        if args.real_layers and lstm is None:
             b = torch.randn(N, generator=gen, device="cuda") * 0.1
             stack.load_weights(l, w, w.half(), b, b.half())
         else:
@@ -375,7 +379,7 @@ def main():
     xs, gs, xs_host, gs_host = [], [], [], []
     # the FP32 gradients entering the top layers arrive as slices of one flat buffer
     tops = [l for l in range(L) if not stack.feeds_next(l)]
-    g_flat = torch.empty(sum(cfg.shapes[l][0] * cfg.shapes[l][2] for l in tops), device="cuda")
+    g_flat = torch.empty(sum(cfg.shapes[l][0] * stack.up_width[l] for l in tops), device="cuda")
     g_off = 0
     for l, (M, K, N) in enumerate(cfg.shapes):
         if chained[l]:
@@ -391,9 +395,10 @@ def main():
         if stack.feeds_next(l):
             gs.append(None); gs_host.append(None)
         else:
-            g = g_flat[g_off:g_off + M * N].view(M, N)
-            g_off += M * N
-            g.copy_(torch.randn(M, N, generator=gen, device="cuda") * cfg.grad_std)
+            Ng = stack.up_width[l]                  # N, or H = N / 4 for an LSTM layer (gradient of h)
+            g = g_flat[g_off:g_off + M * Ng].view(M, Ng)
+            g_off += M * Ng
+            g.copy_(torch.randn(M, Ng, generator=gen, device="cuda") * cfg.grad_std)
             gs.append(g)
             gs_host.append(g.cpu().pin_memory())
     h2d = sum(t.numel() * t.element_size() for t in xs_host + gs_host if t is not None)
@@ -552,8 +557,9 @@ def main():
         "config": {"workload": cfg.name + ": " + cfg.note, "layers": L, "params": cfg.n_params(),
                    "gemm_gflop_per_step": flops_step / 1e9, "optimizer": cfg.optimizer,
                    "parallelism": f"dp{world}" if world > 1 else "single",
-                   "layers_kind": "bias + activation (fused epilogues) + bias gradients" if args.real_layers
-                                  else "plain linear",
+                   "layers_kind": ("LSTM cells on the gate products" if lstm is not None else
+                                   "bias + activation (fused epilogues) + bias gradients" if args.real_layers
+                                   else "plain linear"),
                    "cache": "per-step working set (weights, moments, activations) far exceeds the 126 MB L2"},
         "e2e": {"value": e2e_val, "unit": "TFLOP/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": ms_e2e / args.steps,

@@ -1,6 +1,11 @@
 // LSTM cell (forward and backward) for the gate product of the GNMT-like layers: elementwise,
 // HBM-streaming kernels.  Gates and states are FP16 in memory; the cell is evaluated in FP32
-// (sigma(x) = 1 / (1 + exp(-x)), tanh) and every output is rounded to FP16 once.  Gate order
+// (sigma(x) = 1 / (1 + exp(-x)), tanh) and every output is rounded to FP16 once.  Eight
+// sigma / tanh evaluations per hidden unit (forward three and two, backward the same again):
+// with the library's exactly rounded division and its expf / tanhf the kernels were bound by
+// instruction issue at a third of the HBM rate, so sigma and tanh use the hardware's
+// exponential and reciprocal approximations (a few FP32 units in the last place, far inside
+// half an FP16 unit), with tanh's small-argument and saturated ranges handled apart.  Gate order
 // in the 4H columns of the gate matrix: i, f, g, o.  Each thread handles 8 hidden units of one
 // row with 128-bit loads and stores.
 
@@ -37,7 +42,18 @@ __device__ __forceinline__ void store8(uint16_t* p, const H8& x) {
   __stcs(reinterpret_cast<uint4*>(p), make_uint4(w[0], w[1], w[2], w[3]));
 }
 
-__device__ __forceinline__ float sigm(float x) { return __fdiv_rn(1.0f, __fadd_rn(1.0f, expf(-x))); }
+__device__ __forceinline__ float sigm(float x) { return __fdividef(1.0f, 1.0f + __expf(-x)); }
+
+// tanh(x): x (1 - x^2 / 3) below 0.02 (the next term, 2 x^5 / 15, is under 3e-8 of x there, and
+// the exponential form would cancel); +-1 beyond 9 (tanh(9) rounds to 1 in FP32); else
+// (e^{2|x|} - 1) / (e^{2|x|} + 1) with the sign of x.  NaN falls through to the last form.
+__device__ __forceinline__ float tanh_fast(float x) {
+  const float ax = fabsf(x);
+  if (ax < 0.02f) return x * (1.0f - x * x * (1.0f / 3.0f));
+  if (ax > 9.0f) return copysignf(1.0f, x);
+  const float t = __expf(2.0f * ax);
+  return copysignf(__fdividef(t - 1.0f, t + 1.0f), x);
+}
 
 __global__ void __launch_bounds__(kThreads)
 mp_lstm_cell_fwd_kernel(const uint16_t* __restrict__ G, int64_t ldg, const uint16_t* __restrict__ c_prev,
@@ -51,10 +67,10 @@ mp_lstm_cell_fwd_kernel(const uint16_t* __restrict__ G, int64_t ldg, const uint1
     H8 cn, hh;
 #pragma unroll
     for (int k = 0; k < 8; ++k) {
-      const float i = sigm(gi.v[k]), f = sigm(gf.v[k]), gt = tanhf(gg.v[k]), o = sigm(go.v[k]);
+      const float i = sigm(gi.v[k]), f = sigm(gf.v[k]), gt = tanh_fast(gg.v[k]), o = sigm(go.v[k]);
       const float c = __fadd_rn(__fmul_rn(f, cp.v[k]), __fmul_rn(i, gt));
       cn.v[k] = c;
-      hh.v[k] = __fmul_rn(o, tanhf(c));
+      hh.v[k] = __fmul_rn(o, tanh_fast(c));
     }
     store8(c_new + m * H + j, cn);
     store8(h + m * H + j, hh);
@@ -77,8 +93,8 @@ mp_lstm_cell_bwd_kernel(const uint16_t* __restrict__ G, int64_t ldg, const uint1
     H8 di, df, dg, dout, dcp;
 #pragma unroll
     for (int k = 0; k < 8; ++k) {
-      const float i = sigm(gi.v[k]), f = sigm(gf.v[k]), gt = tanhf(gg.v[k]), o = sigm(go.v[k]);
-      const float tc = tanhf(cn.v[k]);
+      const float i = sigm(gi.v[k]), f = sigm(gf.v[k]), gt = tanh_fast(gg.v[k]), o = sigm(go.v[k]);
+      const float tc = tanh_fast(cn.v[k]);
       float dc = __fmul_rn(__fmul_rn(dhv.v[k], o), __fsub_rn(1.0f, __fmul_rn(tc, tc)));
       if (dc_in != nullptr) dc = __fadd_rn(dc, dci.v[k]);
       di.v[k] = __fmul_rn(__fmul_rn(dc, gt), __fmul_rn(i, __fsub_rn(1.0f, i)));
@@ -96,12 +112,17 @@ mp_lstm_cell_bwd_kernel(const uint16_t* __restrict__ G, int64_t ldg, const uint1
   }
 }
 
-int grid_for(int64_t threads_needed) {
-  int dev = 0, sms = 148;
+// One resident round of blocks (what fits on the device at the kernel's register use): a grid
+// a little larger than that runs a nearly empty second round.
+template <class K>
+int grid_for(K kernel, int64_t threads_needed) {
+  int dev = 0, sms = 148, per_sm = 1;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kThreads, 0);
+  if (per_sm < 1) per_sm = 1;
   const int64_t blocks = (threads_needed + kThreads - 1) / kThreads;
-  const int64_t cap = (int64_t)sms * 8;
+  const int64_t cap = (int64_t)sms * per_sm;
   return (int)(blocks < cap ? (blocks > 0 ? blocks : 1) : cap);
 }
 
@@ -124,7 +145,7 @@ int mp_lstm_cell_fwd(const void* G16, int64_t ldg, const void* c_prev16, void* c
     return mp::set_error(MP_ERR_INVALID_ARG, "mp_lstm_cell_fwd: null pointer");
   if (!mp::aligned16(G16) || !mp::aligned16(c_prev16) || !mp::aligned16(c_new16) || !mp::aligned16(h16))
     return mp::set_error(MP_ERR_ALIGNMENT, "mp_lstm_cell_fwd: pointers must be 16-byte aligned");
-  mp_lstm_cell_fwd_kernel<<<grid_for(M * (H / 8)), kThreads, 0, (cudaStream_t)stream>>>(
+  mp_lstm_cell_fwd_kernel<<<grid_for(mp_lstm_cell_fwd_kernel, M * (H / 8)), kThreads, 0, (cudaStream_t)stream>>>(
       (const uint16_t*)G16, ldg, (const uint16_t*)c_prev16, (uint16_t*)c_new16, (uint16_t*)h16, M, H);
   mp::count_launch();
   MP_CUDA_TRY(cudaGetLastError());
@@ -141,7 +162,7 @@ int mp_lstm_cell_bwd(const void* G16, int64_t ldg, const void* c_prev16, const v
       !mp::aligned16(dh16) || !mp::aligned16(dG16) || !mp::aligned16(dc_prev16) ||
       (dc_in16 && !mp::aligned16(dc_in16)))
     return mp::set_error(MP_ERR_ALIGNMENT, "mp_lstm_cell_bwd: 16-byte alignment and lddg %% 8 == 0 required");
-  mp_lstm_cell_bwd_kernel<<<grid_for(M * (H / 8)), kThreads, 0, (cudaStream_t)stream>>>(
+  mp_lstm_cell_bwd_kernel<<<grid_for(mp_lstm_cell_bwd_kernel, M * (H / 8)), kThreads, 0, (cudaStream_t)stream>>>(
       (const uint16_t*)G16, ldg, (const uint16_t*)c_prev16, (const uint16_t*)c_new16, (const uint16_t*)dh16,
       (const uint16_t*)dc_in16, (uint16_t*)dG16, lddg, (uint16_t*)dc_prev16, M, H);
   mp::count_launch();

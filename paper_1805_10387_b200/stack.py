@@ -24,14 +24,23 @@ class LinearStack:
     def __init__(self, shapes, chained, optimizer="adam", lr=1e-3, beta1=0.9, beta2=0.999,
                  eps=1e-8, momentum=0.9, weight_decay=0.0, init_scale=65536.0,
                  growth_interval=1000, min_scale=1.0, max_scale=2.0 ** 24, dynamic=True,
-                 device="cuda", acts=None, clip=20.0, bias=False, overflow_tolerance=1):
+                 device="cuda", acts=None, clip=20.0, bias=False, overflow_tolerance=1, lstm=None):
         """acts[l]: mp.MP_ACT_* after layer l's product (a layer whose output feeds no chained
-        layer must have MP_ACT_NONE); bias: every layer gets a bias vector."""
+        layer must have MP_ACT_NONE); bias: every layer gets a bias vector; lstm[l]: layer l's
+        product is the gate pre-activation of an LSTM cell (N = 4 H, gate order i, f, g, o): the
+        cell kernels turn it and the cell state c_prev[l] into c_new[l] and h[l], the gradient
+        entering the layer is that of h ([M, H]), and the cell's backward kernel produces the
+        gate gradient that the layer's two backward products consume."""
         self.shapes = [tuple(s) for s in shapes]
         self.chained = list(chained)
         self.L = len(shapes)
         self.acts = list(acts) if acts is not None else [mp.MP_ACT_NONE] * self.L
         self.clip, self.has_bias = float(clip), bool(bias)
+        self.lstm = list(lstm) if lstm is not None else [False] * self.L
+        for l in range(self.L):
+            if self.lstm[l]:
+                assert self.shapes[l][2] % 32 == 0 and self.acts[l] == mp.MP_ACT_NONE and not self.has_bias
+                assert not (l + 1 < self.L and self.chained[l + 1]), "an LSTM layer's gates feed no other layer"
         for l in range(self.L):
             feeds = l + 1 < self.L and self.chained[l + 1]
             assert feeds or self.acts[l] == mp.MP_ACT_NONE, "a top layer has no activation"
@@ -84,20 +93,31 @@ class LinearStack:
         # Scaled upstream gradients of the top layers whose rows need no padding share one flat
         # buffer (ascending layer order): when their FP32 gradients arrive as consecutive slices
         # of one buffer too, a single scaling call covers all of them.
+        # (For an LSTM layer the scaled gradient is that of h, [M, H]; its gate gradient has a
+        # buffer of its own.)
+        self.up_width = [n // 4 if self.lstm[l] else n for l, (_, _, n) in enumerate(self.shapes)]
         self.flat_tops = [l for l in range(self.L) if not (l + 1 < self.L and self.chained[l + 1])
-                          and self.shapes[l][2] % 8 == 0]
-        self.dy_top_flat = torch.zeros(sum(self.shapes[l][0] * self.shapes[l][2] for l in self.flat_tops), **f16)
+                          and self.up_width[l] % 8 == 0]
+        self.dy_top_flat = torch.zeros(sum(self.shapes[l][0] * self.up_width[l] for l in self.flat_tops), **f16)
         flat_off = {}
         o = 0
         for l in self.flat_tops:
             flat_off[l] = o
-            o += self.shapes[l][0] * self.shapes[l][2]
+            o += self.shapes[l][0] * self.up_width[l]
+        self.c_prev, self.c_new, self.h, self.dh, self.dc_prev = ([None] * self.L for _ in range(5))
         for l in range(self.L):
             if self.chained[l]:
                 self.x[l] = self.y[l - 1]
             feeds = l + 1 < self.L and self.chained[l + 1]
             if feeds:
                 self.dy[l] = self.dx[l + 1]
+            elif self.lstm[l]:
+                m, _, n = self.shapes[l]
+                hh = n // 4
+                self.dy[l] = torch.zeros(m, n, **f16)
+                self.dh[l] = self.dy_top_flat[flat_off[l]:flat_off[l] + m * hh].view(m, hh)
+                self.c_prev[l], self.c_new[l], self.h[l], self.dc_prev[l] = (torch.zeros(m, hh, **f16)
+                                                                             for _ in range(4))
             elif l in flat_off:
                 m, _, n = self.shapes[l]
                 self.dy[l] = self.dy_top_flat[flat_off[l]:flat_off[l] + m * n].view(m, n)
@@ -277,7 +297,7 @@ class LinearStack:
             t = gs[l]
             if (t.dtype != torch.float32 or not t.is_contiguous() or t.storage_offset() != off
                     or t.untyped_storage().data_ptr() != store.data_ptr()
-                    or t.numel() != self.shapes[l][0] * self.shapes[l][2]):
+                    or t.numel() != self.shapes[l][0] * self.up_width[l]):
                 return None
             off += t.numel()
         return torch.empty(0, dtype=torch.float32, device=first.device).set_(
@@ -296,13 +316,16 @@ class LinearStack:
             if len(g) > 1 and len({self.x[l].stride(0) for l in g}) == 1:
                 self._call("fwd", mp.mp_linear_fwd_grouped, [Xv(l) for l in g], [self.W16(l) for l in g],
                            [self.Y(l) for l in g], self.workspace)
-                continue
+            else:
+                for l in g:
+                    if self.acts[l] == mp.MP_ACT_NONE and not self.has_bias:
+                        self._call("fwd", mp.mp_linear_fwd, Xv(l), self.W16(l), self.Y(l), self.workspace)
+                    else:
+                        self._call("fwd", mp.mp_linear_fwd_act, Xv(l), self.W16(l), self.b16[l], self.Y(l),
+                                   self.acts[l], self.clip, self.workspace)
             for l in g:
-                if self.acts[l] == mp.MP_ACT_NONE and not self.has_bias:
-                    self._call("fwd", mp.mp_linear_fwd, Xv(l), self.W16(l), self.Y(l), self.workspace)
-                else:
-                    self._call("fwd", mp.mp_linear_fwd_act, Xv(l), self.W16(l), self.b16[l], self.Y(l),
-                               self.acts[l], self.clip, self.workspace)
+                if self.lstm[l]:      # gates -> new cell state and hidden state
+                    self._call("cell", mp.mp_lstm_cell_fwd, self.Y(l), self.c_prev[l], self.c_new[l], self.h[l])
         g_flat = self._flat_upstream(gs)
         if g_flat is not None:        # one scaling call for all flat top layers
             self._call("scale", mp.mp_scale_upstream, g_flat, self.dy_top_flat, self.state)
@@ -310,13 +333,19 @@ class LinearStack:
             for l in reversed(g):
                 if not self.feeds_next(l) and not (g_flat is not None and l in self.flat_tops):
                     n = self.shapes[l][2]
-                    if self.dy[l].shape[1] == n:
+                    if self.lstm[l]:
+                        self._call("scale", mp.mp_scale_upstream, gs[l], self.dh[l], self.state)
+                    elif self.dy[l].shape[1] == n:
                         self._call("scale", mp.mp_scale_upstream, gs[l], self.dy[l], self.state)
                     elif self.only is None or "scale" in self.only:
                         # padded rows: scale into a dense buffer, then place (copy only)
                         tmp = torch.empty(self.shapes[l][0], n, dtype=torch.float16, device=self.device)
                         mp.mp_scale_upstream(gs[l], tmp, self.state)
                         self.dy[l][:, :n].copy_(tmp)
+            for l in reversed(g):
+                if self.lstm[l]:      # gradient of h -> gradient of the gate pre-activations
+                    self._call("cell", mp.mp_lstm_cell_bwd, self.Y(l), self.c_prev[l], self.c_new[l], self.dh[l],
+                               None, self.dY(l), self.dc_prev[l])
             if (len(g) > 1 and len({self.x[l].stride(0) for l in g}) == 1
                     and len({self.dy[l].stride(0) for l in g}) == 1):
                 self._call("wgrad", mp.mp_linear_bwd_wgrad_grouped, [Xv(l) for l in g], [self.dY(l) for l in g],
@@ -368,11 +397,11 @@ class HostPipeline:
 
         def mk_gs():      # one flat FP32 buffer, sliced per top layer: the step scales it in one call
             tops = [l for l in range(s.L) if not s.feeds_next(l)]
-            flat = torch.zeros(sum(s.shapes[l][0] * s.shapes[l][2] for l in tops), dtype=torch.float32,
+            flat = torch.zeros(sum(s.shapes[l][0] * s.up_width[l] for l in tops), dtype=torch.float32,
                                device=s.device)
             out, o = [None] * s.L, 0
             for l in tops:
-                m, _, n = s.shapes[l]
+                m, n = s.shapes[l][0], s.up_width[l]
                 out[l] = flat[o:o + m * n].view(m, n)
                 o += m * n
             return out

@@ -139,7 +139,7 @@ def test_lstm_cell_forward_and_backward(orc, mp, M, H):
     mp.mp_lstm_cell_fwd(Gd, cd, cn, h)
     wc, wh = orc.lstm_cell_fwd(G, c)
 
-    def close(got_bits, want_bits, frac=0.995, scale=None):
+    def close(got_bits, want_bits, frac=0.995, scale=None, extra=None):
         g = got_bits.view(np.float16).astype(np.float64); w = want_bits.view(np.float16).astype(np.float64)
         fin = np.isfinite(w)
         assert (np.isfinite(g) == fin).all()
@@ -148,9 +148,16 @@ def test_lstm_cell_forward_and_backward(orc, mp, M, H):
             # factors like 1 - sigma(x) cancel: an FP32 ulp of sigma is an absolute, not a
             # relative, error of the factor, so allow 1e-5 of the incoming gradient's size
             tol = tol + 1e-5 * np.tile(scale, (1, w.shape[1] // scale.shape[1]))
+        if extra is not None:
+            tol = tol + extra
         assert (np.abs(g - w)[fin] <= tol[fin]).all()
-        assert (got_bits == want_bits).mean() >= frac
-    close(_bits(cn), wc); close(_bits(h), wh)
+        # share of identical bits; on a handful of outputs one differing rounding must not decide
+        assert (got_bits == want_bits).mean() >= frac - 2.0 / got_bits.size
+    # c = f c_prev + i g can cancel: the two sides' sigma and tanh differ by a few FP32 units in
+    # the last place (different exponential and division routines), an absolute error of up to
+    # 4e-6 (|c_prev| + 1) in c and, through tanh' <= 1, in h
+    slack = 4e-6 * (np.abs(c.view(np.float16).astype(np.float64)) + 1.0)
+    close(_bits(cn), wc, extra=slack); close(_bits(h), wh, extra=slack)
     # backward, fed with the oracle's stored c_new so that both sides see identical inputs
     dh = _h(rng.standard_normal((M, H)) * 64); dci = _h(rng.standard_normal((M, H)) * 64)
     dG = _out(M, 4 * H); dcp = torch.empty(M, H, dtype=torch.float16, device="cuda")

@@ -294,6 +294,50 @@ def test_one_scaling_call_over_a_flat_gradient_buffer(orc, mp):
     a.close(); b.close()
 
 
+def test_lstm_gate_layers(orc, mp):
+    """Two independent LSTM gate layers (grouped products, cell kernels wired into the step):
+    every stage of the step is checked against the oracle applied to the operands the GPU stage
+    read -- gate product, cell forward, scaling, cell backward, weight and data gradients."""
+    from paper_1805_10387_b200.stack import LinearStack
+    M, K, H = 96, 64, 32
+    shapes = [(M, K, 4 * H)] * 2
+    rng = np.random.default_rng(21)
+    ws = [rng.standard_normal((K, 4 * H)).astype(np.float32) / np.sqrt(K) for _ in shapes]
+    st = LinearStack(shapes, [False, False], lr=1e-3, init_scale=256.0, growth_interval=1000, lstm=[True, True])
+    assert st.groups == [[0, 1]]
+    for l, w in enumerate(ws):
+        st.load_weights(l, torch.from_numpy(w).cuda(), torch.from_numpy(w).cuda().half())
+        st.c_prev[l].copy_(torch.from_numpy(rng.standard_normal((M, H)).astype(np.float32)).cuda().half())
+    xs = [torch.from_numpy(rng.standard_normal((M, K)).astype(np.float32)).cuda().half() for _ in shapes]
+    gs = [torch.from_numpy((rng.standard_normal((M, H)) * 1e-2).astype(np.float32)).cuda() for _ in shapes]
+
+    def close(got_bits, want_bits, what, scale=None):
+        g, w = _f(got_bits), _f(want_bits)
+        tol = 2.0 ** -10 * np.abs(w) + 2.0 ** -24
+        if scale is not None:
+            tol = tol + 1e-5 * np.tile(scale, (1, w.shape[1] // scale.shape[1]))
+        assert (np.abs(g - w) <= tol).all(), what
+    for step in range(2):
+        w16 = [_bits(st.W16(l)) for l in range(2)]        # the weights this step's products read
+        st.step(xs, gs)
+        torch.cuda.synchronize()
+        for l in range(2):
+            X = _bits(xs[l]); G = _bits(st.Y(l)); cp = _bits(st.c_prev[l])
+            forced_ok(orc, "fwd", X, w16[l], G, ("gates", step, l))
+            wc, wh = orc.lstm_cell_fwd(G, cp)
+            close(_bits(st.c_new[l]), wc, ("c_new", step, l)); close(_bits(st.h[l]), wh, ("h", step, l))
+            dh = _bits(st.dh[l])
+            assert (dh == orc.scale_upstream(gs[l].cpu().numpy(), 256.0)).all()
+            wG, wcp = orc.lstm_cell_bwd(G, cp, _bits(st.c_new[l]), dh, None)
+            sc = np.abs(_f(dh))
+            close(_bits(st.dY(l)), wG, ("dG", step, l), sc); close(_bits(st.dc_prev[l]), wcp, ("dc_prev", step, l), sc)
+            forced_ok(orc, "wgrad", X, _bits(st.dY(l)), _bits(st.dW(l)), ("dW", step, l))
+            forced_ok(orc, "dgrad", _bits(st.dY(l)), w16[l], _bits(st.dX(l)), ("dX", step, l))
+    h = st.state.read()
+    assert h.step == 2 and h.skipped == 0 and h.t == 2
+    st.close()
+
+
 def test_host_pipeline_equals_serial_host_steps(orc, mp):
     """Batches fed from pinned host memory through the double-buffered pipeline (copy of batch
     i+1 under the step of batch i, one CUDA graph per staging set) leave bit-for-bit the state
