@@ -94,6 +94,41 @@ def test_layer_products_at_full_size(orc, mp, name, layer, seed, S):
     st.close()
 
 
+@pytest.mark.parametrize("name,first", [("c2", 0), ("c3", 2)])
+def test_grouped_layer_products_at_full_size(orc, mp, name, first):
+    """The launch configuration the benchmark times for independent layers: four layers of one
+    shape per launch (c2: gate products 0..3; c3: the four projections of block 0).  Every
+    problem's three products are checked on sampled outputs, and the flag against a scan."""
+    cfg = synth.config(name)
+    layers = list(range(first, first + 4))
+    M, K, N = cfg.shapes[first]
+    assert all(cfg.shapes[l] == (M, K, N) for l in layers) and mp.mp_max_group() >= 4
+    S = 2.0 ** 15
+    st = mp.State(init_scale=S)
+    Xs = [synth.activations(cfg, l, 0) for l in layers]
+    Ws = [synth.fp16_bits(synth.weights(cfg, l)).reshape(K, N) for l in layers]
+    dYs = [orc.scale_upstream(synth.upstream(cfg, l, 0), S) for l in layers]
+    Xd, Wd, dYd = [_dev16(x) for x in Xs], [_dev16(w) for w in Ws], [_dev16(d) for d in dYs]
+    mk = lambda r, c: [torch.zeros(r, c, dtype=torch.float16, device="cuda") for _ in layers]
+    Yd, dWd, dXd = mk(M, N), mk(K, N), mk(M, K)
+    need = max(mp.mp_gemm_workspace_bytes_grouped(4, M, K, N, op) for op in (0, 1, 2))
+    ws = torch.empty(max(need, 16), dtype=torch.uint8, device="cuda")
+    mp.mp_linear_fwd_grouped(Xd, Wd, Yd, ws)
+    mp.mp_linear_bwd_wgrad_grouped(Xd, dYd, dWd, st, ws)
+    mp.mp_linear_bwd_dgrad_grouped(dYd, Wd, dXd, ws)
+    torch.cuda.synchronize()
+    assert mp.mp_gemm_device_status() == 0
+    any_inf = 0
+    for i, l in enumerate(layers):
+        same = [_check_samples(orc, "fwd", Xs[i], Ws[i], _bits(Yd[i]), 600, 10 * l),
+                _check_samples(orc, "wgrad", Xs[i], dYs[i], _bits(dWd[i]), 600, 10 * l + 1),
+                _check_samples(orc, "dgrad", dYs[i], Ws[i], _bits(dXd[i]), 600, 10 * l + 2)]
+        assert min(same) > 0.9, (l, same)
+        any_inf |= int(((_bits(dWd[i]) & 0x7C00) == 0x7C00).any())
+    assert st.read().found_inf == any_inf
+    st.close()
+
+
 @pytest.mark.parametrize("P,n_tensors,steps", [(1_000_000, 1, 8), (10_000_000, 8, 8),
                                                (100_000_000, 64, 5), (1_000_000_000, 500, 3)])
 def test_update_sweep_at_full_size(orc, mp, P, n_tensors, steps):
