@@ -190,6 +190,12 @@ int mp_linear_bwd_wgrad_grouped(int count, const void* const* X16, int64_t ldx, 
                                 int64_t lddy, void* const* dW16, int64_t lddw, int64_t M, int64_t K,
                                 int64_t N, mp_state* state, void* workspace, size_t workspace_bytes,
                                 void* stream);
+/* The grouped forward product with the bias and activation of mp_linear_fwd_act: bias16 is a
+ * host array of `count` device pointers (or NULL for no bias), one activation for all. */
+int mp_linear_fwd_act_grouped(int count, const void* const* X16, int64_t ldx, const void* const* W16,
+                              int64_t ldw, const void* const* bias16, void* const* Y16, int64_t ldy,
+                              int64_t M, int64_t K, int64_t N, int act, float clip, void* workspace,
+                              size_t workspace_bytes, void* stream);
 /* Largest `count` the grouped calls take. */
 int mp_max_group(void);
 

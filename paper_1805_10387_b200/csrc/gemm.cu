@@ -81,7 +81,7 @@ struct GemmParams {
   // then the activation.  Data-gradient flavour: zero the output where the layer input
   // mask[row, col] (the previous layer's activated FP16 output) is outside the activation's
   // linear range.  act: 0 none, 1 max(x,0), 2 min(max(x,0),clip).
-  const uint16_t* bias;
+  const uint16_t* bias[MAX_GROUP];   // per problem (all set or all null)
   const uint16_t* mask;
   int64_t ldmask;
   int act;
@@ -197,27 +197,28 @@ __device__ __forceinline__ void finish_chunk(const GemmParams& p, uint32_t (&r)[
                                              bool row_ok, int lane, uint8_t* slot, int half,
                                              const uint32_t* pass_bits, int c, uint32_t& flag_acc,
                                              int prob) {
-  if (FUSED && (p.bias != nullptr || (p.act != 0 && p.mask == nullptr))) {
+  const uint16_t* bias = FUSED ? p.bias[prob] : nullptr;
+  if (FUSED && (bias != nullptr || (p.act != 0 && p.mask == nullptr))) {
     // forward flavour, on the FP32 values: + bias, then the activation
     uint32_t bw[16];                          // 32 bias values as packed halves (0 if absent)
-    if (p.bias != nullptr && col0 + 32 <= p.No) {
+    if (bias != nullptr && col0 + 32 <= p.No) {
 #pragma unroll
       for (int j = 0; j < 4; ++j) {           // same address in every thread: one broadcast load
-        const uint4 q4 = __ldg(reinterpret_cast<const uint4*>(p.bias + col0) + j);
+        const uint4 q4 = __ldg(reinterpret_cast<const uint4*>(bias + col0) + j);
         bw[4 * j] = q4.x; bw[4 * j + 1] = q4.y; bw[4 * j + 2] = q4.z; bw[4 * j + 3] = q4.w;
       }
     } else {
 #pragma unroll
       for (int j = 0; j < 16; ++j) {
-        const uint32_t lo = (p.bias != nullptr && col0 + 2 * j < p.No) ? __ldg(p.bias + col0 + 2 * j) : 0u;
-        const uint32_t hi = (p.bias != nullptr && col0 + 2 * j + 1 < p.No) ? __ldg(p.bias + col0 + 2 * j + 1) : 0u;
+        const uint32_t lo = (bias != nullptr && col0 + 2 * j < p.No) ? __ldg(bias + col0 + 2 * j) : 0u;
+        const uint32_t hi = (bias != nullptr && col0 + 2 * j + 1 < p.No) ? __ldg(bias + col0 + 2 * j + 1) : 0u;
         bw[j] = lo | (hi << 16);
       }
     }
 #pragma unroll
     for (int j = 0; j < 32; ++j) {
       float x = __uint_as_float(r[j]);
-      if (p.bias != nullptr) {
+      if (bias != nullptr) {
         const uint16_t hb = (uint16_t)((j & 1) ? (bw[j >> 1] >> 16) : (bw[j >> 1] & 0xFFFFu));
         x = __fadd_rn(x, __half2float(__ushort_as_half(hb)));
       }
@@ -905,7 +906,8 @@ int choose_splits(int64_t Mo, int64_t No, int64_t R, int64_t count = 1) {
 int64_t ws_ld_for(int64_t No) { return (No + 3) / 4 * 4; }
 
 struct Fuse {
-  const void* bias = nullptr;
+  const void* bias = nullptr;          // single problem
+  const void* const* biases = nullptr; // grouped call: one per problem (overrides `bias`)
   const void* mask = nullptr;
   int64_t ldmask = 0;
   int act = 0;
@@ -919,13 +921,23 @@ struct Operand {
   int64_t mn, red;    // extents along the output dimension and the reduction
 };
 
+// The per-kernel set-up below (shared-memory opt-in, cluster occupancy) is a property of the
+// device the call runs on, so it is remembered per device index.
+constexpr int kMaxDevicesCached = 64;
+int current_device_slot() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0) dev = 0;
+  return dev % kMaxDevicesCached;
+}
+
 template <bool A_MN, bool B_MN, bool WIDE>
 int launch(const GroupMaps& maps, const GemmParams& p, int grid, cudaStream_t st) {
-  static bool attr_set = false;
-  if (!attr_set) {
+  static bool attr_set[kMaxDevicesCached] = {};
+  const int slot = current_device_slot();
+  if (!attr_set[slot]) {
     MP_CUDA_TRY(cudaFuncSetAttribute(mp_gemm_kernel<A_MN, B_MN, WIDE>,
                                      cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
-    attr_set = true;
+    attr_set[slot] = true;
   }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(grid, 1, 1);
@@ -944,7 +956,8 @@ int launch(const GroupMaps& maps, const GemmParams& p, int grid, cudaStream_t st
 
 template <bool A_MN, bool B_MN, bool WIDE>
 int launch_pair(const GroupMaps& maps, const GemmParams& p, int64_t work, cudaStream_t st) {
-  static int max_pairs = 0;
+  static int max_pairs_of[kMaxDevicesCached] = {};
+  int& max_pairs = max_pairs_of[current_device_slot()];
   if (max_pairs == 0) {
     MP_CUDA_TRY(cudaFuncSetAttribute(mp_gemm_pair_kernel<A_MN, B_MN, WIDE>,
                                      cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM2_BYTES));
@@ -1015,12 +1028,15 @@ int run_gemm(const char* name, int count, const Operand* As, const Operand* Bs, 
   p.n_tiles = (int)((No + BN - 1) / BN);
   p.num_kb = (int)((R + BK - 1) / BK);
   p.m_fast = Mo < No ? 1 : 0;
-  const bool fused = fuse.bias != nullptr || fuse.act != 0;
-  if (fused && count != 1)
-    return mp::set_error(MP_ERR_INVALID_ARG, "%s: the fused epilogues take one problem per call", name);
+  const bool has_bias = fuse.bias != nullptr || fuse.biases != nullptr;
+  const bool fused = has_bias || fuse.act != 0;
+  if (fuse.mask != nullptr && count != 1)
+    return mp::set_error(MP_ERR_INVALID_ARG, "%s: the masked data gradient takes one problem per call", name);
   p.splits = fused ? 1 : choose_splits(Mo, No, R, count);   // the fused epilogue needs the whole sum
   p.work_per_problem = p.m_tiles * p.n_tiles * p.splits;
-  p.bias = (const uint16_t*)fuse.bias; p.mask = (const uint16_t*)fuse.mask;
+  for (int i = 0; i < MAX_GROUP; ++i)
+    p.bias[i] = (const uint16_t*)(fuse.biases ? fuse.biases[i < count ? i : 0] : fuse.bias);
+  p.mask = (const uint16_t*)fuse.mask;
   p.ldmask = fuse.ldmask; p.act = fuse.act; p.clip = fuse.clip;
   for (int i = 0; i < MAX_GROUP; ++i) p.out[i] = (uint16_t*)outs[i < count ? i : 0];
   p.ldo = ldo;
@@ -1278,6 +1294,26 @@ int mp_linear_fwd_act(const void* X16, int64_t ldx, const void* W16, int64_t ldw
   Fuse f;
   f.bias = bias16; f.act = act; f.clip = clip;
   return run_gemm("mp_linear_fwd_act", A, B, Y16, ldy, nullptr, false, workspace, workspace_bytes,
+                  (cudaStream_t)stream, f);
+}
+
+int mp_linear_fwd_act_grouped(int count, const void* const* X16, int64_t ldx, const void* const* W16,
+                              int64_t ldw, const void* const* bias16, void* const* Y16, int64_t ldy,
+                              int64_t M, int64_t K, int64_t N, int act, float clip, void* workspace,
+                              size_t workspace_bytes, void* stream) {
+  if (int rc = check_act("mp_linear_fwd_act_grouped", act, clip)) return rc;
+  if (count < 1 || count > MAX_GROUP || !X16 || !W16 || !Y16)
+    return mp::set_error(MP_ERR_INVALID_ARG, "mp_linear_fwd_act_grouped: 1..%d problems, non-null arrays", MAX_GROUP);
+  if (bias16) {
+    for (int i = 0; i < count; ++i)
+      if (!bias16[i] || !mp::aligned16(bias16[i]))
+        return mp::set_error(MP_ERR_ALIGNMENT, "mp_linear_fwd_act_grouped: every bias must be non-null and 16-byte aligned");
+  }
+  Operand A[MAX_GROUP], B[MAX_GROUP];
+  for (int i = 0; i < count; ++i) { A[i] = Operand{X16[i], ldx, false, M, K}; B[i] = Operand{W16[i], ldw, true, N, K}; }
+  Fuse f;
+  f.biases = bias16; f.act = act; f.clip = clip;
+  return run_gemm("mp_linear_fwd_act_grouped", count, A, B, Y16, ldy, nullptr, false, workspace, workspace_bytes,
                   (cudaStream_t)stream, f);
 }
 

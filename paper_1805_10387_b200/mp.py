@@ -64,6 +64,8 @@ SIGNATURES = {
     "mp_linear_fwd_grouped": (_i32, [_i32, _p, _i64, _p, _i64, _p, _i64, _i64, _i64, _i64, _p, _sz, _p]),
     "mp_linear_bwd_dgrad_grouped": (_i32, [_i32, _p, _i64, _p, _i64, _p, _i64, _i64, _i64, _i64, _p, _sz, _p]),
     "mp_linear_bwd_wgrad_grouped": (_i32, [_i32, _p, _i64, _p, _i64, _p, _i64, _i64, _i64, _i64, _p, _p, _sz, _p]),
+    "mp_linear_fwd_act_grouped": (_i32, [_i32, _p, _i64, _p, _i64, _p, _p, _i64, _i64, _i64, _i64, _i32,
+                                         C.c_float, _p, _sz, _p]),
     "mp_max_group": (_i32, []),
     "mp_gemm_workspace_bytes_grouped": (_sz, [_i32, _i64, _i64, _i64, _i32]),
     "mp_linear_fwd_act": (_i32, [_p, _i64, _p, _i64, _p, _p, _i64, _i64, _i64, _i64, _i32, C.c_float, _p, _sz, _p]),
@@ -213,6 +215,18 @@ def mp_linear_fwd_grouped(X16s, W16s, Y16s, workspace=None):
     assert K2 == K and ys == (M, N) and len(X16s) == len(W16s) == len(Y16s)
     ws, nb = _ws(workspace)
     _check(lib().mp_linear_fwd_grouped(len(X16s), x, ldx, w, ldw, y, ldy, M, K, N, ws, nb, _stream()))
+
+
+def mp_linear_fwd_act_grouped(X16s, W16s, bias16s, Y16s, act=MP_ACT_NONE, clip=20.0, workspace=None):
+    (x, ldx, (M, K)), (w, ldw, (K2, N)), (y, ldy, ys) = _mats(X16s), _mats(W16s), _mats(Y16s)
+    assert K2 == K and ys == (M, N) and len(X16s) == len(W16s) == len(Y16s)
+    b = None
+    if bias16s is not None:
+        assert len(bias16s) == len(X16s) and all(t.numel() == N and t.is_contiguous() for t in bias16s)
+        b = (C.c_void_p * len(bias16s))(*[_dev(t, torch.float16) for t in bias16s])
+    ws, nb = _ws(workspace)
+    _check(lib().mp_linear_fwd_act_grouped(len(X16s), x, ldx, w, ldw, b, y, ldy, M, K, N, act, clip, ws, nb,
+                                           _stream()))
 
 
 def mp_linear_bwd_dgrad_grouped(dY16s, W16s, dX16s, workspace=None):

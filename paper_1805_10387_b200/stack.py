@@ -124,13 +124,13 @@ class LinearStack:
             else:
                 self.dy[l] = torch.zeros(self.shapes[l][0], _align(self.shapes[l][2]), **f16)
         # Runs of consecutive layers that depend on nothing in the stack (no chained input, output
-        # feeding no layer), have one shape and plain epilogues go to the grouped calls, a few
+        # feeding no layer), have one shape and no activation go to the grouped calls, a few
         # layers per launch; every other layer is a group of one.
         self.groups = []
         gmax = mp.mp_max_group()
         for l in range(self.L):
             free = (not self.chained[l] and not (l + 1 < self.L and self.chained[l + 1])
-                    and self.acts[l] == mp.MP_ACT_NONE and not self.has_bias)
+                    and self.acts[l] == mp.MP_ACT_NONE)
             g = self.groups[-1] if self.groups else None
             if (free and g is not None and g[1] and len(g[0]) < gmax
                     and self.shapes[g[0][0]] == self.shapes[l]):
@@ -314,8 +314,13 @@ class LinearStack:
         Xv = lambda l: self.x[l][:, :self.shapes[l][1]]
         for g in self.groups:
             if len(g) > 1 and len({self.x[l].stride(0) for l in g}) == 1:
-                self._call("fwd", mp.mp_linear_fwd_grouped, [Xv(l) for l in g], [self.W16(l) for l in g],
-                           [self.Y(l) for l in g], self.workspace)
+                if self.has_bias:
+                    self._call("fwd", mp.mp_linear_fwd_act_grouped, [Xv(l) for l in g], [self.W16(l) for l in g],
+                               [self.b16[l] for l in g], [self.Y(l) for l in g], mp.MP_ACT_NONE, self.clip,
+                               self.workspace)
+                else:
+                    self._call("fwd", mp.mp_linear_fwd_grouped, [Xv(l) for l in g], [self.W16(l) for l in g],
+                               [self.Y(l) for l in g], self.workspace)
             else:
                 for l in g:
                     if self.acts[l] == mp.MP_ACT_NONE and not self.has_bias:
@@ -350,6 +355,9 @@ class LinearStack:
                     and len({self.dy[l].stride(0) for l in g}) == 1):
                 self._call("wgrad", mp.mp_linear_bwd_wgrad_grouped, [Xv(l) for l in g], [self.dY(l) for l in g],
                            [self.dW(l) for l in g], self.state, self.workspace)
+                if self.has_bias:
+                    for l in reversed(g):
+                        self._call("bgrad", mp.mp_bias_grad, self.dY(l), self.db[l], self.state, self.workspace)
                 self._call("dgrad", mp.mp_linear_bwd_dgrad_grouped, [self.dY(l) for l in g],
                            [self.W16(l) for l in g], [self.dX(l) for l in g], self.workspace)
                 continue

@@ -77,6 +77,25 @@ def test_dgrad_activation_mask_integer_exact(orc, mp, act, M, K, N):
         assert (want == 0).mean() > 0.3
 
 
+@pytest.mark.parametrize("act", ["none", "relu"])
+def test_grouped_fwd_bias_activation_integer_exact(orc, mp, act):
+    """Three problems with their own biases in one launch: integer operands, bit-exact against the
+    oracle's forward product with bias and activation."""
+    M, K, N = 300, 72, 264
+    rng = np.random.default_rng(31)
+    Xs = [_h(rng.integers(-2, 3, (M, K))) for _ in range(3)]
+    Ws = [_h(rng.integers(-2, 3, (K, N))) for _ in range(3)]
+    bs = [_h(rng.integers(-3, 4, (N,))) for _ in range(3)]
+    Ys = [_out(M, N) for _ in range(3)]
+    bd = [torch.from_numpy(b.view(np.float16).copy()).cuda() for b in bs]
+    mp.mp_linear_fwd_act_grouped([_dev(x) for x in Xs], [_dev(w) for w in Ws], bd, Ys,
+                                 {"none": mp.MP_ACT_NONE, "relu": mp.MP_ACT_RELU}[act], 20.0)
+    torch.cuda.synchronize()
+    assert mp.mp_gemm_device_status() == 0
+    for i in range(3):
+        assert (_bits(Ys[i]) == orc.linear_fwd_act(Xs[i], Ws[i], bs[i], act)).all(), i
+
+
 def test_fwd_act_random_values_within_tolerance(orc, mp):
     rng = np.random.default_rng(1)
     M, K, N = 384, 520, 264
