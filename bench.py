@@ -36,7 +36,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # dram__bytes_write.sum, mean over one step's product launches; on c2 a launch holds four layers'
 # products, 4 x 95.4 MB algorithmic), keyed by workload, valid only for the kernel source it was
 # taken on.
-NCU_TRAFFIC = {"sha": "735224e192c28da6", "bytes_per_launch": {"c2": 402.2e6}}
+NCU_TRAFFIC = {"sha": "735224e192c28da6", "bytes_per_launch": {"c2": 401.4e6}}
 
 
 def peaks():
