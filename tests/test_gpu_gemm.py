@@ -155,6 +155,45 @@ def test_grouped_call_equals_single_calls(orc, mp, op, M, K, N, count):
     st.close()
 
 
+@pytest.mark.parametrize("M,K,N,count", [(520, 200, 264, 3), (2048, 512, 1024, 4)])
+def test_grouped_call_is_bitwise_the_single_call_on_random_values(mp, M, K, N, count):
+    """A tile is accumulated in the same order whether its problem is launched alone or in a
+    group, so with random operands the grouped outputs equal the single calls' bit for bit
+    wherever both split the reduction the same way (always for these forward and data-gradient
+    products; for the weight gradient when the scratch sizes say the split counts agree)."""
+    g = torch.Generator(device="cuda"); g.manual_seed(M + count)
+    X = [torch.randn(M, K, generator=g, device="cuda").half() for _ in range(count)]
+    W = [(torch.randn(K, N, generator=g, device="cuda") / 16).half() for _ in range(count)]
+    dY = [(torch.randn(M, N, generator=g, device="cuda") * 4).half() for _ in range(count)]
+    z = lambda r, c: [torch.zeros(r, c, dtype=torch.float16, device="cuda") for _ in range(count)]
+    need = max(max(mp.mp_gemm_workspace_bytes_grouped(count, M, K, N, op), mp.mp_gemm_workspace_bytes(M, K, N, op))
+               for op in range(3))
+    ws = torch.empty(max(need, 16), dtype=torch.uint8, device="cuda")
+    Yg, dXg, dWg, Ys, dXs, dWs = z(M, N), z(M, K), z(K, N), z(M, N), z(M, K), z(K, N)
+    mp.mp_linear_fwd_grouped(X, W, Yg, ws)
+    mp.mp_linear_bwd_dgrad_grouped(dY, W, dXg, ws)
+    mp.mp_linear_bwd_wgrad_grouped(X, dY, dWg, None, ws)
+    for i in range(count):
+        mp.mp_linear_fwd(X[i], W[i], Ys[i], ws)
+        mp.mp_linear_bwd_dgrad(dY[i], W[i], dXs[i], ws)
+        mp.mp_linear_bwd_wgrad(X[i], dY[i], dWs[i], None, ws)
+    torch.cuda.synchronize()
+    assert mp.mp_gemm_device_status() == 0
+    same_split = {op: mp.mp_gemm_workspace_bytes_grouped(count, M, K, N, op) == count * mp.mp_gemm_workspace_bytes(M, K, N, op)
+                  for op in range(3)}
+    for i in range(count):
+        if same_split[0]:
+            assert torch.equal(Yg[i].view(torch.int16), Ys[i].view(torch.int16))
+        if same_split[1]:
+            assert torch.equal(dXg[i].view(torch.int16), dXs[i].view(torch.int16))
+        if same_split[2]:
+            assert torch.equal(dWg[i].view(torch.int16), dWs[i].view(torch.int16))
+        else:   # another fixed order of FP32 partial sums: equal to within an FP16 rounding
+            a, b = dWg[i].float(), dWs[i].float()
+            assert (a - b).abs().max() <= 2.0 ** -9 * b.abs().max()
+    assert same_split[0] and same_split[1]
+
+
 def test_grouped_call_rejects_bad_counts(mp):
     a = torch.zeros(16, 16, dtype=torch.float16, device="cuda")
     n = mp.mp_max_group()
