@@ -84,6 +84,9 @@ INT_CASES = [
     (300, 200, 520),    # several tiles in both directions, ragged tails
     (260, 1000, 130),   # long reduction, many ring wraps
     (129, 72, 257),     # one past a tile edge
+    (8, 20000, 8),      # very long reduction on a sliver of output (split paths, 313 k-blocks)
+    (5000, 8, 8),       # many row tiles, one partial k-block
+    (16, 8, 3000),      # many column tiles
 ]
 
 
