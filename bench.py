@@ -39,6 +39,16 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 NCU_TRAFFIC = {"sha": "735224e192c28da6", "bytes_per_launch": {"c2": 401.4e6}}
 
 
+# DRAM bytes per parameter of the fused update from one ncu capture at 1e8 parameters in 64 tensors
+# (2.7400 GB per launch); a launch over P parameters moves P times this (traffic grows in
+# proportion: every parameter is touched once), valid only for the kernel source it was taken on.
+NCU_UPDATE_TRAFFIC = {"sha": "d29d336f54d27289", "bytes_per_param": 27.40}
+
+
+def update_kernel_sha():
+    return hashlib.sha256(open(os.path.join(ROOT, "paper_1805_10387_b200", "csrc", "update.cu"), "rb").read()).hexdigest()[:16]
+
+
 def peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -241,7 +251,10 @@ def run_update_sweep(args):
         "gpu_launches": int(mp.mp_kernel_launch_count() - launches0),
         "roofline": {"kernel": "mp_master_update_kernel", "bound": "hbm", "achieved": top["gbs_28B"],
                      "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": top["gbs_28B"] / pk["hbm_gbs"],
-                     "traffic": None, "peak_source": pk_src + " copy", "frac_of_nominal_8000": top["gbs_28B"] / 8000.0},
+                     "traffic": (NCU_UPDATE_TRAFFIC["bytes_per_param"] * top["params"]
+                                 if NCU_UPDATE_TRAFFIC["sha"] == update_kernel_sha() else None),
+                     "traffic_note": "ncu capture at 1e8 parameters scaled by the parameter count",
+                     "peak_source": pk_src + " copy", "frac_of_nominal_8000": top["gbs_28B"] / 8000.0},
         "sweep": rows, "clocks": clocks}))
 
 
