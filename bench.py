@@ -71,13 +71,13 @@ class ClockSampler:
          "clocks_event_reasons.sw_power_cap")
 
     def __init__(self, index):
-        self.rows, self.proc, self.index = [], None, index
+        self.rows, self.times, self.proc, self.index = [], [], None, index
 
     def start(self):
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
         except OSError:
@@ -86,19 +86,31 @@ class ClockSampler:
     def _read(self):
         for line in self.proc.stdout:
             self.rows.append([c.strip() for c in line.split(",")])
+            self.times.append(time.time())
 
-    def stop(self):
+    def stop(self, window=None):
+        """window = (t0, t1) in time.time() seconds: `sm_mhz` is then the median over the samples
+        that arrived inside it (the device-timed regions), and `sm_mhz_all` the median over the
+        whole run, which also holds the PCIe-bound end-to-end region."""
         if not self.proc:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         self.proc.terminate()
         self.thread.join(timeout=2)
-        sm = sorted(float(r[0]) for r in self.rows if r and r[0].replace(".", "").isdigit())
+        ok = lambda r: r and r[0].replace(".", "").isdigit()
+        sm_all = sorted(float(r[0]) for r in self.rows if ok(r))
+        sm = sm_all
+        if window is not None:
+            inside = sorted(float(r[0]) for r, t in zip(self.rows, self.times)
+                            if ok(r) and window[0] <= t <= window[1] + 0.05)
+            if inside:
+                sm = inside
         mx = [float(r[1]) for r in self.rows if len(r) > 1 and r[1].replace(".", "").isdigit()]
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         reasons = [n for i, n in enumerate(names) if any(len(r) > 3 + i and r[3 + i] == "Active" for r in self.rows)]
         pw = [float(r[2]) for r in self.rows if len(r) > 2 and r[2].replace(".", "").isdigit()]
         return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": mx[0] if mx else None,
-                "reasons": reasons, "samples": len(sm), "power_w_max": max(pw) if pw else None}
+                "reasons": reasons, "samples": len(sm), "power_w_max": max(pw) if pw else None,
+                "sm_mhz_all": sm_all[len(sm_all) // 2] if sm_all else None, "samples_all": len(sm_all)}
 
 
 # ------------------------------------------------------------------ reference arm (CPU oracle)
@@ -457,6 +469,7 @@ def main():
         run_step()
     torch.cuda.synchronize()
     st0 = stack.state.read()
+    t_dev0 = time.time()
     ms_total = timed(run_step, args.steps)
     st1 = stack.state.read()
     launches = launches_per_step * args.steps
@@ -505,6 +518,7 @@ def main():
             per.setdefault(name, []).append(a.elapsed_time(b))
         timed_how = ("a second timed region of the same steps, launched call by call with a CUDA-event "
                      "pair around every launch")
+    t_dev1 = time.time()
     # (C) end to end: pinned host inputs in, loss-scale state out, every step
     # through the double-buffered host pipeline: the copies of batch i+1 run under the kernels of
     # batch i; every step still copies its inputs in and reads the state back
@@ -530,7 +544,7 @@ def main():
     if dist is not None:
         dist.all_reduce(ms_e2e_t, op=dist.ReduceOp.MAX)
     ms_e2e = float(ms_e2e_t.item())
-    clocks = sampler.stop() if rank == 0 else None
+    clocks = sampler.stop((t_dev0, t_dev1)) if rank == 0 else None
     assert mp.mp_gemm_device_status() == 0, "a GEMM kernel reported a device-side error"
 
     flops_step = cfg.gemm_flops()
