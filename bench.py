@@ -4,6 +4,10 @@
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2|c3|c4|c5] [--impl reference]
   python bench.py --workload c3 --per-shape      (each layer shape's products alone, beside cuBLAS)
 
+Without --workload the line's top-level fields are the GNMT-like stack (c2) and the other
+workloads (c3, c4, and the update-only sweep c5 up to 1e9 parameters) are timed after it with
+fewer steps and reported under `workloads`, each with its own `roofline`.
+
 One step = forward, weight-gradient and data-gradient products of every layer (FP16 operands,
 FP32 accumulation), upstream scaling, the fused unscale / inspect / FP32-master optimizer /
 FP16 recast update and the loss-scale state machine, on one batch of seeded synthetic input.
@@ -37,6 +41,8 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # products, 4 x 95.4 MB algorithmic), keyed by workload, valid only for the kernel source it was
 # taken on.
 NCU_TRAFFIC = {"sha": "735224e192c28da6", "bytes_per_launch": {"c2": 401.4e6}}
+# flop per clock and SM of the FP16 tensor pipe (one 128 x 256 x 16 MMA per SM in 128 clocks)
+TENSOR_FLOP_PER_CLK_SM = 8192
 
 
 # DRAM bytes per parameter of the fused update from one ncu capture at 1e8 parameters in 64 tensors
@@ -65,10 +71,12 @@ def kernel_sha():
 
 
 class ClockSampler:
-    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    """Samples nvidia-smi clocks and throttle reasons while the timed regions run; every sample
+    keeps its arrival time so that a region can ask for the samples that fell inside it."""
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
          "clocks_event_reasons.sw_power_cap")
+    NAMES = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
 
     def __init__(self, index):
         self.rows, self.times, self.proc, self.index = [], [], None, index
@@ -88,36 +96,37 @@ class ClockSampler:
             self.rows.append([c.strip() for c in line.split(",")])
             self.times.append(time.time())
 
-    def stop(self, window=None):
-        """window = (t0, t1) in time.time() seconds: `sm_mhz` is then the median over the samples
-        that arrived inside it (the device-timed regions), and `sm_mhz_all` the median over the
-        whole run, which also holds the PCIe-bound end-to-end region."""
+    def stop(self):
+        if self.proc:
+            self.proc.terminate()
+            self.thread.join(timeout=2)
+
+    @staticmethod
+    def _num(r, i):
+        return float(r[i]) if len(r) > i and r[i].replace(".", "").isdigit() else None
+
+    def summary(self, windows=None):
+        """windows: list of (t0, t1) in time.time() seconds; `sm_mhz` is the median over the samples
+        inside them (all samples when None or when none fell inside)."""
         if not self.proc:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        self.proc.terminate()
-        self.thread.join(timeout=2)
-        ok = lambda r: r and r[0].replace(".", "").isdigit()
-        sm_all = sorted(float(r[0]) for r in self.rows if ok(r))
-        sm = sm_all
-        if window is not None:
-            inside = sorted(float(r[0]) for r, t in zip(self.rows, self.times)
-                            if ok(r) and window[0] <= t <= window[1] + 0.05)
-            if inside:
-                sm = inside
-        mx = [float(r[1]) for r in self.rows if len(r) > 1 and r[1].replace(".", "").isdigit()]
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        reasons = [n for i, n in enumerate(names) if any(len(r) > 3 + i and r[3 + i] == "Active" for r in self.rows)]
-        pw = [float(r[2]) for r in self.rows if len(r) > 2 and r[2].replace(".", "").isdigit()]
+        rows = list(zip(self.rows, self.times))
+        inside = [r for r, t in rows if windows and any(a <= t <= b + 0.05 for a, b in windows)]
+        use = inside if inside else [r for r, _ in rows]
+        sm = sorted(x for x in (self._num(r, 0) for r in use) if x is not None)
+        mx = [x for x in (self._num(r, 1) for r in use) if x is not None]
+        pw = [x for x in (self._num(r, 2) for r in use) if x is not None]
+        reasons = [n for i, n in enumerate(self.NAMES) if any(len(r) > 3 + i and r[3 + i] == "Active" for r in use)]
         return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": mx[0] if mx else None,
                 "reasons": reasons, "samples": len(sm), "power_w_max": max(pw) if pw else None,
-                "sm_mhz_all": sm_all[len(sm_all) // 2] if sm_all else None, "samples_all": len(sm_all)}
+                "power_w_median": sorted(pw)[len(pw) // 2] if pw else None}
 
 
 # ------------------------------------------------------------------ reference arm (CPU oracle)
 def oracle_sample_step(orc, synth, cfg, rows, upd_params, data=None):
     """One bounded sample of the workload on the CPU oracle: the three products of layer 0 on
     its first `rows` rows and the optimizer update of `upd_params` parameters.  Returns
-    (seconds, gemm_flops, update_bytes, data)."""
+    (seconds of the products, seconds of the update, gemm_flops, update_bytes, data)."""
     import numpy as np
     M, K, N = cfg.shapes[0]
     if data is None:
@@ -136,6 +145,7 @@ def oracle_sample_step(orc, synth, cfg, rows, upd_params, data=None):
     dY = orc.scale_upstream(g, S)
     dW = orc.linear_bwd_wgrad(X, dY)
     orc.linear_bwd_dgrad(dY, W16)
+    t1 = time.perf_counter()
     n = st["w32"].size
     g16 = np.ascontiguousarray(dW.reshape(-1)[:n])
     if not orc.found_inf(dW):
@@ -143,8 +153,27 @@ def oracle_sample_step(orc, synth, cfg, rows, upd_params, data=None):
             orc.adam_update(g16, st["w32"], st["m"], st["v"], st["w16"], S, cfg.lr, cfg.beta1, cfg.beta2, cfg.eps, 1)
         else:
             orc.momentum_update(g16, st["w32"], st["m"], st["w16"], S, cfg.lr, cfg.momentum)
-    dt = time.perf_counter() - t0
-    return dt, 3 * 2 * rows * K * N, n * (28 if cfg.optimizer == "adam" else 20), data
+    t2 = time.perf_counter()
+    return t1 - t0, t2 - t1, 3 * 2 * rows * K * N, n * (28 if cfg.optimizer == "adam" else 20), data
+
+
+def cpu_baseline_of(orc, synth, cfg, seconds):
+    """The oracle as it stands on the host cores, on a bounded sample of the workload: products and
+    update timed apart (GFLOP/s, GB/s) and together (`value`, the whole-sample analogue of the
+    GPU line's `value`)."""
+    rows, upd = 64, 1 << 21
+    tg = tu = 0.0
+    fl = by = 0
+    data = None
+    t_budget = time.perf_counter()
+    while tg + tu < seconds and time.perf_counter() - t_budget < 3.5 * seconds:
+        a, b, f, nb, data = oracle_sample_step(orc, synth, cfg, rows, upd, data)
+        tg, tu, fl, by = tg + a, tu + b, fl + f, by + nb
+    return {"value": fl / (tg + tu) / 1e12, "unit": "TFLOP/s", "cores": orc.hardware_threads(), "kind": "oracle",
+            "gemm_gflops": fl / tg / 1e9, "update_gbs": by / tu / 1e9,
+            "update_note": "the oracle's update loop is one thread (a plain loop, as it stands)",
+            "sample": f"fwd+wgrad+dgrad of layer 0 of {cfg.name} on its first {rows} rows + update of {upd} params, "
+                      f"repeated for {tg + tu:.1f} s"}
 
 
 def run_reference(args):
@@ -154,22 +183,24 @@ def run_reference(args):
     from oracle import mp_oracle as orc
     from paper_1805_10387_b200 import synth
     orc.build()
-    cfg = synth.config("c2" if args.workload == "c5" else args.workload)
+    wl = args.workload or "c2"
+    cfg = synth.config("c2" if wl == "c5" else wl)
     # size the per-step sample so that the whole run (warm-up + steps) takes about two minutes
     upd = 1 << 20
     data = None
-    dt, _, _, data = oracle_sample_step(orc, synth, cfg, 8, upd, data)
-    dt, _, _, data = oracle_sample_step(orc, synth, cfg, 8, upd, data)
+    a, b, _, _, data = oracle_sample_step(orc, synth, cfg, 8, upd, data)
+    a, b, _, _, data = oracle_sample_step(orc, synth, cfg, 8, upd, data)
     budget = 120.0 / max(1, args.steps + args.warmup)
-    rows = int(max(4, min(64, 8 * budget / max(dt, 1e-3))))
+    rows = int(max(4, min(64, 8 * budget / max(a + b, 1e-3))))
     data = None
     for _ in range(args.warmup):
-        _, _, _, data = oracle_sample_step(orc, synth, cfg, rows, upd, data)
-    tot, flops = 0.0, 0
+        _, _, _, _, data = oracle_sample_step(orc, synth, cfg, rows, upd, data)
+    tg = tu = 0.0
+    flops = nbytes = 0
     for _ in range(args.steps):
-        dt, f, _, data = oracle_sample_step(orc, synth, cfg, rows, upd, data)
-        tot += dt
-        flops += f
+        a, b, f, nb, data = oracle_sample_step(orc, synth, cfg, rows, upd, data)
+        tg, tu, flops, nbytes = tg + a, tu + b, flops + f, nbytes + nb
+    tot = tg + tu
     val = flops / tot / 1e12
     cores = orc.hardware_threads()
     sample = f"per step: fwd+wgrad+dgrad of layer 0 on its first {rows} rows + update of {upd} params"
@@ -178,27 +209,44 @@ def run_reference(args):
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": tot / args.steps * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f16 in / f32 accumulate",
         "data": "synthetic", "config": {"workload": cfg.name + ": " + cfg.note},
-        "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": sample,
+                         "gemm_gflops": flops / tg / 1e9, "update_gbs": nbytes / tu / 1e9},
         "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
 
 
+def settle(fn, seconds, sync):
+    """Runs fn back to back, untimed, for about `seconds` of wall time so that the timed region
+    that follows starts in the power and clock state the same work settles into."""
+    t0 = time.time()
+    n = 0
+    while time.time() - t0 < seconds:
+        for _ in range(8):
+            fn()
+        n += 8
+        sync()
+    return time.time() - t0
+
+
 # ------------------------------------------------------------------ update-only sweep
-def run_update_sweep(args):
+def run_update_sweep(args, sampler=None, steps=None, settle_s=1.0):
     """Update-only workload: unscale / inspect / Adam / FP16 recast over 1e6 .. 1e9 parameters in
     1 .. 500 tensors of log-uniform sizes, gradients rn16(S * N(0, 1e-3)).  Per size: GB/s on the
     algorithmic 28 B/param for applied steps with the flag trusted (check_mode 0) and with the
-    in-call inspection (check_mode 1, 30 B/param moved), and the time of a skipped step."""
+    in-call inspection (check_mode 1, 30 B/param moved), and the time of a skipped step.  Every
+    timed loop follows `settle_s` seconds of the same launches, untimed.  Returns the JSON object."""
     import torch
     from paper_1805_10387_b200 import mp, synth
-    if int(os.environ.get("RANK", "0")) != 0:
-        return
     torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
     mp.lib()
+    steps = steps or args.steps
     pk, pk_src = peaks()
     rows = []
-    sampler = ClockSampler(0)
-    sampler.start()
+    own_sampler = sampler is None
+    if own_sampler:
+        sampler = ClockSampler(int(os.environ.get("LOCAL_RANK", "0")))
+        sampler.start()
+    windows = []
     launches0 = mp.mp_kernel_launch_count()
     for P, n in ((1_000_000, 1), (10_000_000, 8), (100_000_000, 64), (1_000_000_000, 500)):
         if P > args.max_params:
@@ -222,13 +270,15 @@ def run_update_sweep(args):
             k = min(blk, tot - lo)
             g16[lo:lo + k] = z[:k].half()
             w32[lo:lo + k] = z[:k] * 1e-4
-        iters = max(3, min(args.steps, int(2e10 // (P * 30)) + 3))
+        iters = max(3, min(steps, int(2e10 // (P * 30)) + 3))
+
+        def one(mode):
+            mp.mp_master_update(plan, st, opt, mode)
+            mp.mp_loss_scale_update(st)
 
         def timed(mode, reps):
-            for _ in range(3):
-                mp.mp_master_update(plan, st, opt, mode)
-                mp.mp_loss_scale_update(st)
-            torch.cuda.synchronize()
+            settle(lambda: one(mode), settle_s, torch.cuda.synchronize)
+            t0 = time.time()
             ts = []
             for _ in range(reps):
                 a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -238,36 +288,45 @@ def run_update_sweep(args):
                 mp.mp_loss_scale_update(st)
                 ts.append((a, b))
             torch.cuda.synchronize()
+            if P >= 100_000_000:
+                windows.append((t0, time.time()))
             return sum(a.elapsed_time(b) for a, b in ts) / reps
         ms0 = timed(0, iters)
         ms1 = timed(1, iters)
+        skipped0 = st.read().skipped
         g16.view(torch.int16)[offs[-1] + counts[-1] - 1] = 0x7C00      # overflow: skipped steps
         ms_skip = timed(1, iters)
-        assert st.read().skipped >= iters
+        assert st.read().skipped - skipped0 >= iters
         rows.append({"params": P, "tensors": n, "ms_trusted_flag": ms0, "gbs_28B": P * 28 / ms0 / 1e6,
+                     "frac_of_peak": P * 28 / ms0 / 1e6 / pk["hbm_gbs"],
                      "ms_with_inspection": ms1, "gbs_28B_with_inspection": P * 28 / ms1 / 1e6,
                      "gbs_30B_moved_with_inspection": P * 30 / ms1 / 1e6, "ms_skipped_step": ms_skip,
+                     "timed_launches": iters,
                      "note": "L2-resident / launch-bound" if P * 16 < 126e6 else "HBM-bound"})
         plan.close()
         st.close()
         del g16, w16, w32, m, v, z
         torch.cuda.empty_cache()
-    clocks = sampler.stop()
+    if own_sampler:
+        sampler.stop()
+    clocks = sampler.summary(windows)
     top = rows[-1]
-    print(json.dumps({
-        "metric": METRIC, "value": top["gbs_28B"], "unit": "GB/s", "n_gpus": 1, "steps": args.steps,
+    return {
+        "metric": METRIC, "value": top["gbs_28B"], "unit": "GB/s", "n_gpus": 1, "steps": steps,
         "warmup": 3, "ms_per_step": top["ms_trusted_flag"], "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f16 gradients / f32 master", "data": "synthetic",
         "config": {"workload": "c5: update-only sweep, Adam, 1e6..1e9 parameters in 1..500 log-uniform tensors",
-                   "cache": "1e8 and 1e9 parameters (1.6 / 16 GB of state) far exceed the 126 MB L2"},
+                   "cache": "1e8 and 1e9 parameters (1.6 / 16 GB of state) far exceed the 126 MB L2",
+                   "settle_s": settle_s},
         "gpu_launches": int(mp.mp_kernel_launch_count() - launches0),
         "roofline": {"kernel": "mp_master_update_kernel", "bound": "hbm", "achieved": top["gbs_28B"],
                      "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": top["gbs_28B"] / pk["hbm_gbs"],
                      "traffic": (NCU_UPDATE_TRAFFIC["bytes_per_param"] * top["params"]
                                  if NCU_UPDATE_TRAFFIC["sha"] == update_kernel_sha() else None),
                      "traffic_note": "ncu capture at 1e8 parameters scaled by the parameter count",
+                     "algorithmic_bytes_per_launch": 28 * top["params"], "avg_launch_ms": top["ms_trusted_flag"],
                      "peak_source": pk_src + " copy", "frac_of_nominal_8000": top["gbs_28B"] / 8000.0},
-        "sweep": rows, "clocks": clocks}))
+        "sweep": rows, "clocks": clocks}
 
 
 # ------------------------------------------------------------------ per-shape timing
@@ -335,46 +394,18 @@ def run_per_shape(args):
     print(json.dumps({"per_shape": rows, "workload": cfg.name, "launches_per_graph": reps}))
 
 
-# ------------------------------------------------------------------ CUDA arm
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
-    ap.add_argument("--warmup", type=int, default=10)
-    ap.add_argument("--workload", default="c2", choices=["c2", "c3", "c4", "c5"])
-    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
-    ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--real-layers", action="store_true",
-                    help="biases on every layer and an activation inside every chain (ReLU; clipped ReLU for c4)")
-    ap.add_argument("--per-shape", action="store_true",
-                    help="time each distinct layer shape's three products alone, beside torch.matmul")
-    ap.add_argument("--max-params", type=float, default=1e9, help="c5: largest parameter count of the sweep")
-    args = ap.parse_args()
-    if args.impl == "reference":
-        return run_reference(args)
-    if args.workload == "c5":
-        return run_update_sweep(args)
-    if args.per_shape:
-        return run_per_shape(args)
-
-    import numpy as np
+# ------------------------------------------------------------------ CUDA arm: one stack workload
+def run_stack(args, name, steps, sampler, dist, full):
+    """Times one of the GEMM workloads (c2, c3, c4) and returns its JSON object.  `full`: also the
+    end-to-end region (host inputs) and the CPU baseline.  Every device-timed region is preceded
+    by `--settle` seconds of untimed replays of the same region."""
     import torch
     from paper_1805_10387_b200 import mp, synth
-    from paper_1805_10387_b200.stack import LinearStack
+    from paper_1805_10387_b200.stack import HostPipeline, LinearStack
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
-    torch.cuda.set_device(local)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    mp.lib()
-
-    cfg = synth.config(args.workload)
+    cfg = synth.config(name)
     L = len(cfg.shapes)
     chained = [cfg.chained(l) for l in range(L)]
     acts = None
@@ -384,13 +415,14 @@ def main():
     elif args.real_layers:
         act = mp.MP_ACT_CLIPPED_RELU if cfg.name == "c4" else mp.MP_ACT_RELU
         acts = [act if (l + 1 < L and chained[l + 1]) else mp.MP_ACT_NONE for l in range(L)]
+    comm = None
+    if world > 1:      # data parallel over rows: weights replicated, FP16 weight gradients summed
+        from paper_1805_10387_b200 import dp
+        comm = dp.Comm()
     stack = LinearStack(cfg.shapes, chained, optimizer=cfg.optimizer, lr=cfg.lr, beta1=cfg.beta1,
                         beta2=cfg.beta2, eps=cfg.eps, momentum=cfg.momentum, init_scale=cfg.init_scale,
                         growth_interval=cfg.growth_interval, acts=acts, bias=args.real_layers and lstm is None,
-                        lstm=lstm)
-    if world > 1:      # data parallel over rows: weights replicated, FP16 weight gradients summed
-        from paper_1805_10387_b200 import dp
-        stack.grad_sync = dp.allreduce_gradients
+                        lstm=lstm, comm=comm, shard_update=args.shard_update)
     gen = torch.Generator(device="cuda")
     gen.manual_seed(1234 + cfg.seed)           # same weights on every rank
     for l, (M, K, N) in enumerate(cfg.shapes):
@@ -416,7 +448,7 @@ def main():
             x = torch.zeros(M, (K + 7) // 8 * 8, dtype=torch.float16, device="cuda")
             x[:, :K] = z.half()
             xs.append(x)
-            xs_host.append(x[:, :K].contiguous().cpu().pin_memory())
+            xs_host.append(x[:, :K].contiguous().cpu().pin_memory() if full else None)
         if stack.feeds_next(l):
             gs.append(None); gs_host.append(None)
         else:
@@ -425,7 +457,7 @@ def main():
             g_off += M * Ng
             g.copy_(torch.randn(M, Ng, generator=gen, device="cuda") * cfg.grad_std)
             gs.append(g)
-            gs_host.append(g.cpu().pin_memory())
+            gs_host.append(g.cpu().pin_memory() if full else None)
     h2d = sum(t.numel() * t.element_size() for t in xs_host + gs_host if t is not None)
     d2h = 56
 
@@ -434,139 +466,146 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    def timed(fn, steps):
-        """max over ranks of the device time of `steps` calls, in ms"""
+    windows = {}
+
+    def timed(fn, n, key=None, settle_s=None):
+        """max over ranks of the device time of n calls, in ms, after the settling replays"""
+        s = settle(fn, args.settle if settle_s is None else settle_s, torch.cuda.synchronize)
         barrier()
+        t0 = time.time()
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record()
-        for _ in range(steps):
+        for _ in range(n):
             fn()
         b.record()
         barrier()
+        if key is not None:
+            windows[key] = (t0, time.time())
         ms = torch.tensor([a.elapsed_time(b)], device="cuda")
         if dist is not None:
             dist.all_reduce(ms, op=dist.ReduceOp.MAX)
-        return float(ms.item())
+        return float(ms.item()), s
 
     for _ in range(max(args.warmup, 3)):
         stack.step(xs, gs)
     torch.cuda.synchronize()
-    st0 = stack.state.read()
     launches0 = mp.mp_kernel_launch_count()
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
-        time.sleep(0.3)
     # (A) the step as one CUDA graph replay per step: `value`
-    launches_per_step = mp.mp_kernel_launch_count()
     stack.step(xs, gs)
-    launches_per_step = mp.mp_kernel_launch_count() - launches_per_step
-    use_graph = world == 1          # the data-parallel step (NCCL all-reduce inside) is launched call by call
+    launches_per_step = mp.mp_kernel_launch_count() - launches0
+    use_graph = world == 1          # the data-parallel step (NCCL collectives inside) is launched call by call
     if use_graph:
         stack.capture(xs, gs)
     run_step = stack.replay if use_graph else (lambda: stack.step(xs, gs))
-    for _ in range(3):
-        run_step()
-    torch.cuda.synchronize()
     st0 = stack.state.read()
-    t_dev0 = time.time()
-    ms_total = timed(run_step, args.steps)
+    ms_total, settle_step = timed(run_step, steps, "step")
     st1 = stack.state.read()
-    launches = launches_per_step * args.steps
-    # (B) per-call device times for the roofline.  One GPU: the same step recorded once more with
-    # an event-record node before and after every call; each timed replay is followed at once by
-    # an untimed one, so the device never idles while the host reads the events (a timed replay
-    # runs in the same power and clock state as the steps of (A); the event nodes themselves
-    # stop a kernel's prologue from overlapping its predecessor's tail, so this region is a
-    # little slower than (A) and is not the one `value` is taken from).  Several GPUs: call by
-    # call with an event pair around every launch.
+    launches = launches_per_step * steps
+    # (B) the products alone: the step's forward, weight-gradient and data-gradient calls (same
+    # order, same buffers) recorded without the other calls and without event nodes, replayed
+    # back to back: elapsed device time / launches = the GEMM kernels' average launch duration
+    # with their prologue overlap intact and no event between them.  Then per-call device times
+    # for the breakdown: the step recorded once more with an event-record node before and after
+    # every call, each timed replay followed at once by an untimed one, so that the device never
+    # idles while the host reads the events.  Several GPUs: call by call with event pairs.
     per = {}
     gemm_only = None
+    upd_only = None
     if use_graph:
-        # the products alone: the step's forward, weight-gradient and data-gradient calls (same
-        # order, same buffers) recorded without the other calls and without event nodes, replayed
-        # back to back: elapsed device time / launches = the GEMM kernels' average launch
-        # duration with their prologue overlap intact and no event between them
         gemm_only = {}
-        for key, classes in (("gemm", ("fwd", "dgrad", "wgrad")), ("fwd", ("fwd",)), ("dgrad", ("dgrad",)),
-                             ("wgrad", ("wgrad",))):
+        for key, classes, ss in (("gemm", ("fwd", "dgrad", "wgrad"), None), ("fwd", ("fwd",), args.settle / 4),
+                                 ("dgrad", ("dgrad",), args.settle / 4), ("wgrad", ("wgrad",), args.settle / 4)):
             n0 = mp.mp_kernel_launch_count()
             g_sub = stack.capture_only(xs, gs, classes)
             n_launch = mp.mp_kernel_launch_count() - n0
-            for _ in range(3):
-                g_sub.replay()
-            gemm_only[key] = (timed(g_sub.replay, args.steps) / args.steps, n_launch)
+            ms, s = timed(g_sub.replay, steps, key if key == "gemm" else None, ss)
+            gemm_only[key] = (ms / steps, n_launch, s)
         g_timed, ev = stack.capture_timed(xs, gs)
         done = torch.cuda.Event()
 
         def timed_steps():
-            for _ in range(args.steps):
+            for _ in range(steps):
                 g_timed.replay()
                 done.record()
                 stack.replay()
                 done.synchronize()
-                for name, a, b in ev:
-                    per.setdefault(name, []).append(a.elapsed_time(b))
-        ms_events = timed(timed_steps, 1) / 2.0
-        timed_how = ("a second timed region: the step's graph recorded with an event-record node before and "
+                for nm, a, b in ev:
+                    per.setdefault(nm, []).append(a.elapsed_time(b))
+        settle(stack.replay, args.settle / 2, torch.cuda.synchronize)
+        barrier()
+        a_t, b_t = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a_t.record(); timed_steps(); b_t.record(); barrier()
+        ms_events = a_t.elapsed_time(b_t) / 2.0
+        timed_how = ("a further timed region: the step's graph recorded with an event-record node before and "
                      "after every call, each timed replay followed by an untimed one")
     else:
         stack.events = []
-        ms_events = timed(lambda: stack.step(xs, gs), args.steps)
+        ms_events, _ = timed(lambda: stack.step(xs, gs), steps, None, 0.0)
         events, stack.events = stack.events, None
-        for name, a, b in events:
-            per.setdefault(name, []).append(a.elapsed_time(b))
-        timed_how = ("a second timed region of the same steps, launched call by call with a CUDA-event "
+        for nm, a, b in events:
+            per.setdefault(nm, []).append(a.elapsed_time(b))
+        timed_how = ("a further timed region of the same steps, launched call by call with a CUDA-event "
                      "pair around every launch")
-    t_dev1 = time.time()
-    # (C) end to end: pinned host inputs in, loss-scale state out, every step
-    # through the double-buffered host pipeline: the copies of batch i+1 run under the kernels of
-    # batch i; every step still copies its inputs in and reads the state back
-    from paper_1805_10387_b200.stack import HostPipeline
-    pipe = HostPipeline(stack, use_graph=use_graph)
+    # (C) end to end: pinned host inputs in, loss-scale state out, every step, through the
+    # double-buffered host pipeline: the copies of batch i+1 run under the kernels of batch i
+    ms_e2e = None
+    if full:
+        pipe = HostPipeline(stack, use_graph=use_graph)
 
-    def e2e_steps(n):
-        def go():
-            pipe.submit(xs_host, gs_host)
-            for i in range(n):
-                if i + 1 < n:
-                    pipe.submit(xs_host, gs_host)
-                pipe.run()
-        return go
-    e2e_steps(3)()
-    barrier()
-    a_e, b_e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    a_e.record()
-    e2e_steps(args.steps)()
-    b_e.record()
-    barrier()
-    ms_e2e_t = torch.tensor([a_e.elapsed_time(b_e)], device="cuda")
-    if dist is not None:
-        dist.all_reduce(ms_e2e_t, op=dist.ReduceOp.MAX)
-    ms_e2e = float(ms_e2e_t.item())
-    clocks = sampler.stop((t_dev0, t_dev1)) if rank == 0 else None
+        def e2e_steps(n):
+            def go():
+                pipe.submit(xs_host, gs_host)
+                for i in range(n):
+                    if i + 1 < n:
+                        pipe.submit(xs_host, gs_host)
+                    pipe.run()
+            return go
+        e2e_steps(3)()
+        barrier()
+        t0 = time.time()
+        a_e, b_e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a_e.record()
+        e2e_steps(steps)()
+        b_e.record()
+        barrier()
+        windows["e2e"] = (t0, time.time())
+        ms_e2e_t = torch.tensor([a_e.elapsed_time(b_e)], device="cuda")
+        if dist is not None:
+            dist.all_reduce(ms_e2e_t, op=dist.ReduceOp.MAX)
+        ms_e2e = float(ms_e2e_t.item())
+    # (D) the fused update alone, replayed back to back (last: it moves the weights without new
+    # gradients, which nothing after it reads)
+    if use_graph:
+        n0 = mp.mp_kernel_launch_count()
+        g_upd = stack.capture_only(xs, gs, ("update",))
+        n_launch = mp.mp_kernel_launch_count() - n0
+        ms, s = timed(g_upd.replay, steps, "update", args.settle / 2)
+        upd_only = (ms / steps / max(n_launch, 1), s)
     assert mp.mp_gemm_device_status() == 0, "a GEMM kernel reported a device-side error"
+    assert stack.state.read().status == 0
 
     flops_step = cfg.gemm_flops()
-    ms_step = ms_total / args.steps
+    ms_step = ms_total / steps
     value = world * flops_step / (ms_step * 1e-3) / 1e12
-    e2e_val = world * flops_step / (ms_e2e / args.steps * 1e-3) / 1e12
     pk, pk_src = peaks()
     gemm_calls = sum(len(per.get(k, [])) for k in ("fwd", "dgrad", "wgrad"))
     if gemm_only is not None:
-        gemm_ms = gemm_only["gemm"][0] * args.steps
-        gemm_launches = gemm_only["gemm"][1] * args.steps
+        gemm_ms = gemm_only["gemm"][0] * steps
+        gemm_launches = gemm_only["gemm"][1] * steps
         per_op = {k: (flops_step / 3) / (gemm_only[k][0] * 1e-3) / 1e12 for k in ("fwd", "dgrad", "wgrad")}
         gemm_how = ("the step's product calls alone (same order and buffers, no other call, no event between "
-                    "them) as a CUDA graph replayed back to back for the same number of steps; CUDA events "
-                    "around the region; launches include the split-reduction kernels of the weight gradients")
+                    "them) as a CUDA graph replayed back to back for the same number of steps, after settle_s "
+                    "seconds of the same replays untimed; CUDA events around the region; launches include the "
+                    "split-reduction kernels of the weight gradients")
+        gemm_settle = gemm_only["gemm"][2]
     else:
         gemm_ms = sum(sum(per.get(k, [])) for k in ("fwd", "dgrad", "wgrad"))
         gemm_launches = gemm_calls
-        per_op = {k: (flops_step / 3) * args.steps / (sum(per[k]) * 1e-3) / 1e12
+        per_op = {k: (flops_step / 3) * steps / (sum(per[k]) * 1e-3) / 1e12
                   for k in ("fwd", "dgrad", "wgrad") if k in per}
         gemm_how = timed_how
-    gemm_tflops = flops_step * args.steps / (gemm_ms * 1e-3) / 1e12
+        gemm_settle = 0.0
+    gemm_tflops = flops_step * steps / (gemm_ms * 1e-3) / 1e12
     skipped = st1.skipped - st0.skipped
     bytes_per_param = 28 if cfg.optimizer == "adam" else 20
     upd_ms = per.get("update", [0.0])
@@ -574,67 +613,165 @@ def main():
     # a skipped step's update returns at once (a few microseconds); GB/s is quoted on the
     # applied ones only
     applied_ms = [t for t in upd_ms if t >= 0.25 * max(upd_ms)]
-    upd_gbs = upd_bytes / (sum(applied_ms) / len(applied_ms) * 1e-3) / 1e9
+    upd_ms_in_step = sum(applied_ms) / len(applied_ms)
+    upd_ms_alone = upd_only[0] if upd_only is not None else upd_ms_in_step
+    upd_gbs = upd_bytes / (upd_ms_alone * 1e-3) / 1e9
     sha = kernel_sha()
-    traffic = NCU_TRAFFIC["bytes_per_launch"].get(args.workload) if NCU_TRAFFIC["sha"] == sha else None
+    traffic = NCU_TRAFFIC["bytes_per_launch"].get(name) if NCU_TRAFFIC["sha"] == sha and not args.real_layers else None
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    clk = {k: (sampler.summary([w]) if sampler is not None else None) for k, w in windows.items()}
+    settled = gemm_settle >= 1.5
+    peak = pk["bf16_tflops_sustained"] if settled else pk["bf16_tflops"]
+    gemm_mhz = clk.get("gemm", {}).get("sm_mhz") if clk.get("gemm") else None
+    clock_peak = sms * TENSOR_FLOP_PER_CLK_SM * gemm_mhz * 1e6 / 1e12 if gemm_mhz else None
     out = {
-        "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+        "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f16 in / f32 accumulate", "data": "synthetic",
         "config": {"workload": cfg.name + ": " + cfg.note, "layers": L, "params": cfg.n_params(),
                    "gemm_gflop_per_step": flops_step / 1e9, "optimizer": cfg.optimizer,
-                   "parallelism": f"dp{world}" if world > 1 else "single",
+                   "parallelism": (f"dp{world}" + (" sharded update" if stack.shard_update else "")) if world > 1 else "single",
                    "layers_kind": ("LSTM cells on the gate products" if lstm is not None else
                                    "bias + activation (fused epilogues) + bias gradients" if args.real_layers
                                    else "plain linear"),
-                   "cache": "per-step working set (weights, moments, activations) far exceeds the 126 MB L2"},
-        "e2e": {"value": e2e_val, "unit": "TFLOP/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "ms_per_step": ms_e2e / args.steps,
-                "feed": "two staging sets: batch i+1 is copied from pinned host memory while batch i runs"},
+                   "cache": "per-step working set (weights, moments, activations) far exceeds the 126 MB L2",
+                   "settle_s": settle_step,
+                   "settle": "every device-timed region follows that many seconds of untimed replays of itself"},
         "gpu_launches": int(launches),
         "launch_mode": "one CUDA graph replay per step (captured from the same C-ABI calls)" if use_graph
                        else "call by call",
-        "ms_per_step_in_event_timed_region": ms_events / args.steps,
+        "ms_per_step_in_event_timed_region": ms_events / steps,
         "skipped_steps_in_timed_region": int(skipped),
         "loss_scale": st1.scale,
         "roofline": {"kernel": "mp_gemm_pair_kernel", "bound": "tensor", "achieved": gemm_tflops,
-                     "peak": pk["bf16_tflops_sustained"], "unit": "TFLOP/s",
-                     "frac": gemm_tflops / pk["bf16_tflops_sustained"], "traffic": traffic,
-                     "peak_source": f"{pk_src} cuBLAS bf16 sustained (fp16 nominal ratio 1.0)",
+                     "peak": peak, "unit": "TFLOP/s", "frac": gemm_tflops / peak, "traffic": traffic,
+                     "peak_source": (f"{pk_src} cuBLAS bf16 sustained (the region is timed after {gemm_settle:.1f} s of "
+                                     f"itself; fp16 nominal ratio 1.0)" if settled else
+                                     f"{pk_src} cuBLAS bf16 burst (no settling run; fp16 nominal ratio 1.0)"),
+                     "settle_s": gemm_settle,
                      "frac_of_burst_peak": gemm_tflops / pk["bf16_tflops"],
+                     "frac_of_sustained_peak": gemm_tflops / pk["bf16_tflops_sustained"],
                      "frac_of_nominal_2250": gemm_tflops / 2250.0,
+                     "sm_mhz_in_region": gemm_mhz, "clock_peak_tflops": clock_peak,
+                     "frac_of_clock_peak": gemm_tflops / clock_peak if clock_peak else None,
+                     "clock_peak_how": f"{sms} SMs x {TENSOR_FLOP_PER_CLK_SM} flop/clk x median SM clock sampled inside this region",
                      "launches": gemm_launches, "avg_launch_ms": gemm_ms / max(gemm_launches, 1),
-                     "algorithmic_gflop_per_launch": flops_step * args.steps / max(gemm_launches, 1) / 1e9,
+                     "algorithmic_gflop_per_launch": flops_step * steps / max(gemm_launches, 1) / 1e9,
+                     "algorithmic_mb_per_launch": cfg_gemm_bytes(cfg) * steps / max(gemm_launches, 1) / 1e6,
                      "grouping": "independent same-shape layers run up to four per launch",
                      "calls": gemm_calls, "timed_in": gemm_how,
                      "per_op_tflops": per_op},
         "update": {"kernel": "mp_master_update_kernel", "bound": "hbm", "achieved": upd_gbs,
                    "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": upd_gbs / pk["hbm_gbs"],
                    "frac_of_nominal_8000": upd_gbs / 8000.0, "bytes_per_param": bytes_per_param,
-                   "avg_launch_ms": sum(applied_ms) / len(applied_ms), "peak_source": pk_src + " copy"},
+                   "algorithmic_bytes_per_launch": upd_bytes,
+                   "avg_launch_ms": upd_ms_alone, "peak_source": pk_src + " copy",
+                   "timed_in": ("the step's update call alone as a CUDA graph replayed back to back after settling "
+                                "replays" if upd_only is not None else timed_how),
+                   "in_step": {"avg_launch_ms": upd_ms_in_step, "achieved": upd_bytes / (upd_ms_in_step * 1e-3) / 1e9,
+                               "note": "between event nodes inside the step, right after the products"},
+                   "traffic": (NCU_UPDATE_TRAFFIC["bytes_per_param"] * cfg.n_params()
+                               if NCU_UPDATE_TRAFFIC["sha"] == update_kernel_sha() and cfg.optimizer == "adam" else None)},
         # device time per call class per step from the event-timed region (sum over the step's
         # calls; every call's interval is stretched by its two event nodes, a few microseconds)
         "breakdown_timed_in": timed_how,
-        "breakdown_ms_per_step": {k: sum(v) / args.steps for k, v in sorted(per.items())},
-        "clocks": clocks,
+        "breakdown_ms_per_step": {k: sum(v) / steps for k, v in sorted(per.items())},
+        "clocks": None,
+        "clocks_by_region": clk,
     }
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+    if ms_e2e is not None:
+        out["e2e"] = {"value": world * flops_step / (ms_e2e / steps * 1e-3) / 1e12, "unit": "TFLOP/s",
+                      "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / steps,
+                      "feed": "two staging sets: batch i+1 is copied from pinned host memory while batch i runs"}
+    if sampler is not None:
+        dev_windows = [w for k, w in windows.items() if k != "e2e"]
+        c = sampler.summary(dev_windows)
+        c["regions"] = "median over the device-timed regions (step, products, update); the PCIe-bound e2e region apart"
+        out["clocks"] = c
+    if rank == 0 and world == 1 and full and not args.no_cpu_baseline:
         from oracle import mp_oracle as orc
         orc.build()
-        rows, upd = 64, 1 << 21
-        tot, fl, data = 0.0, 0, None
-        t_budget = time.perf_counter()
-        while tot < 12.0 and time.perf_counter() - t_budget < 40.0:
-            dt, f, _, data = oracle_sample_step(orc, synth, cfg, rows, upd, data)
-            tot += dt
-            fl += f
-        out["cpu_baseline"] = {"value": fl / tot / 1e12, "unit": "TFLOP/s", "cores": orc.hardware_threads(),
-                               "kind": "oracle",
-                               "sample": f"fwd+wgrad+dgrad of layer 0 on its first {rows} rows + update of "
-                                         f"{upd} params, repeated for {tot:.1f} s"}
+        out["cpu_baseline"] = cpu_baseline_of(orc, synth, cfg, 12.0)
+    stack.close()
+    del stack, xs, gs, g_flat
+    torch.cuda.empty_cache()
+    return out
+
+
+def cfg_gemm_bytes(cfg):
+    """Algorithmic bytes of one step's products: every operand read once, every output written once."""
+    return sum(2 * (3 * (m * k + k * n + m * n)) for m, k, n in cfg.shapes)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--workload", default=None, choices=["c2", "c3", "c4", "c5"],
+                    help="time this workload only (default: c2 at the top level, c3, c4 and c5 under `workloads`)")
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--settle", type=float, default=2.0,
+                    help="seconds of untimed replays before each device-timed region (0: none; the roofline "
+                         "then divides by the burst peak)")
+    ap.add_argument("--real-layers", action="store_true",
+                    help="biases on every layer and an activation inside every chain (ReLU; clipped ReLU for c4)")
+    ap.add_argument("--per-shape", action="store_true",
+                    help="time each distinct layer shape's three products alone, beside torch.matmul")
+    ap.add_argument("--shard-update", action="store_true",
+                    help="several GPUs: reduce-scatter the gradients, update a 1/N slice of the master per rank, "
+                         "all-gather the FP16 weights (default: all-reduce and a replicated update)")
+    ap.add_argument("--max-params", type=float, default=1e9, help="c5: largest parameter count of the sweep")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    import torch
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if args.workload == "c5":
+        if rank == 0:
+            print(json.dumps(run_update_sweep(args)))
+        return
+    if args.per_shape:
+        args.workload = args.workload or "c2"
+        return run_per_shape(args)
+
+    from paper_1805_10387_b200 import mp
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    mp.lib()
+    sampler = None
+    if rank == 0:
+        sampler = ClockSampler(local)
+        sampler.start()
+        time.sleep(0.3)
+    main_wl = args.workload or "c2"
+    out = run_stack(args, main_wl, args.steps, sampler, dist, full=True)
+    if args.workload is None and world == 1:
+        # the other workloads, fewer steps, device-timed regions only
+        others = {}
+        n = max(20, args.steps // 4)
+        for wl in ("c3", "c4"):
+            o = run_stack(args, wl, n, sampler, dist, full=False)
+            others[wl] = {k: o[k] for k in ("value", "unit", "steps", "ms_per_step", "config", "gpu_launches",
+                                            "skipped_steps_in_timed_region", "loss_scale", "roofline", "update",
+                                            "breakdown_ms_per_step", "clocks")}
+        o = run_update_sweep(args, sampler, steps=n, settle_s=min(1.0, args.settle))
+        others["c5"] = {k: o[k] for k in ("value", "unit", "ms_per_step", "config", "gpu_launches", "roofline",
+                                          "sweep", "clocks")}
+        out["workloads"] = others
+        out["gpu_launches_all_workloads"] = int(out["gpu_launches"] + sum(w["gpu_launches"] for w in others.values()))
+    if sampler is not None:
+        sampler.stop()
     if rank == 0:
         print(json.dumps(out))
-    stack.close()
     if dist is not None:
         dist.destroy_process_group()
 

@@ -24,6 +24,18 @@
  *   - The library owns only mp_state and mp_update_plan objects.  It runs on the device
  *     that is current when a function is called; objects belong to the device they were
  *     created on.
+ *   - Calls may come from several host threads.  The one-time set-up that a first call does per
+ *     device and per kernel flavour (attribute, occupancy and symbol queries) is serialised
+ *     inside the library; a state or plan object must not be used by two threads at once.
+ *   - Device-side errors.  Every wait inside a kernel is bounded.  A product kernel whose wait
+ *     runs out stops taking work, releases what it holds and returns; it records
+ *     MP_ERR_TIMEOUT in a device-wide status word and, when the call was given a state, in
+ *     state->status.  While either is set, mp_master_update writes nothing and
+ *     mp_loss_scale_update changes nothing (it copies the device-wide word into
+ *     state->status): the training state is frozen as it was before the faulty step.  The host
+ *     learns of it from mp_state_read (status) or mp_gemm_device_status, and resumes with
+ *     mp_gemm_device_status (which clears the device-wide word) followed by mp_state_write
+ *     with status = 0.
  */
 #ifndef MP_H_
 #define MP_H_
@@ -84,9 +96,10 @@ typedef struct {
   int32_t growth_interval, dynamic;
   int32_t good_steps;  /* clean steps since S last changed                                  */
   int32_t found_inf;   /* flag accumulated by the current step so far                       */
-  int32_t status;      /* MP_OK or the first device-side error (MP_ERR_TIMEOUT)             */
+  int32_t status;      /* MP_OK or the first device-side error (MP_ERR_TIMEOUT), see above  */
   int32_t overflow_tolerance;
-  int32_t strikes;     /* overflows since S last changed (always 0 with tolerance 1)        */
+  int32_t strikes;     /* overflows since S last changed (dynamic scale with tolerance 1:
+                          always 0; static scale: S never changes, so every overflow counts) */
   int64_t t;           /* applied optimizer steps                                           */
   int64_t step;        /* all steps                                                         */
   int64_t skipped;     /* overflow steps                                                    */
@@ -156,8 +169,10 @@ int mp_loss_scale_update(mp_state* state, void* stream);
  * allocating library routine.
  *
  * The first call on each device looks up the array's device address (one cheap runtime query,
- * no allocation, done with that device current); make that first call before starting any
- * stream capture.  All calls on a device share the one array: two calls whose kernels may
+ * no allocation, done with that device current), and like every product call the first one per
+ * device and kernel flavour also sets kernel attributes and asks for occupancy; make a first
+ * call with sizes of the same class (K above or at most 128, i.e. the same kernel flavour)
+ * before starting any stream capture.  All calls on a device share the one array: two calls whose kernels may
  * overlap on the GPU (different streams) race on it and must be ordered by the caller.  The
  * array keeps whatever the previous call left; that is harmless because each call overwrites
  * every partial sum it later reads, so nothing has to start at zero. */
@@ -276,6 +291,15 @@ int mp_state_write(mp_state* state, const mp_state_host* in, void* stream);
 int mp_state_read_log(mp_state* state, mp_log_record* out, int max_records, int* n_out,
                       void* stream);
 
+/* Data-parallel runs whose ranks each inspect only a slice of the summed gradients (Section 4
+ * of the paper: replicas that exchange gradients; the sharded-update schedule) agree on the
+ * overflow flag by reducing one word across ranks.  These two calls move the flag between the
+ * device state and a caller-owned int32 device word, asynchronously on `stream`, with no host
+ * round trip: export writes *word = (found_inf != 0); import ORs (*word != 0) into found_inf.
+ * word: device pointer, 4-byte aligned. */
+int mp_state_export_flag(const mp_state* state, int32_t* word, void* stream);
+int mp_state_import_flag(mp_state* state, const int32_t* word, void* stream);
+
 /* Plan over n tensors: g16[i], w16[i] FP16 and w32[i], m[i], v[i] FP32 device buffers of
  * count[i] elements each (count[i] == 0 is legal and skipped).  v may be NULL for a plan
  * used only with momentum (m then holds the momentum buffer).  The pointer arrays are host
@@ -284,6 +308,17 @@ int mp_update_plan_create(int n, void* const* g16, void* const* w32, void* const
                           void* const* v, void* const* w16, const int64_t* count,
                           mp_update_plan** out);
 int mp_update_plan_destroy(mp_update_plan* plan); /* NULL is accepted */
+
+/* Error-path self-test (not one of the step's calls; the paper has no counterpart).  Launches
+ * the forward product's kernel on ONE output tile (M <= 128, N <= 256; arguments otherwise as
+ * mp_linear_fwd) with its loader told to fetch nothing and every pipeline wait limited to
+ * wait_us microseconds (1 .. 2000000).  No copy is ever in flight: the waits run out, the
+ * kernel records MP_ERR_TIMEOUT (device-wide and, if state != NULL, in state->status), frees
+ * its tensor memory and returns without writing Y16.  It exists so that the library's
+ * reaction to an expired wait can be exercised on a healthy GPU. */
+int mp_selftest_wait_timeout(const void* X16, int64_t ldx, const void* W16, int64_t ldw, void* Y16,
+                             int64_t ldy, int64_t M, int64_t K, int64_t N, int64_t wait_us,
+                             mp_state* state, void* stream);
 
 /* Synchronises the device and reports in *out the first device-side error recorded by a GEMM
  * kernel since the last call (MP_OK, or MP_ERR_TIMEOUT when a bounded wait on a pipeline

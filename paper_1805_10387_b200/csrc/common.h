@@ -29,6 +29,9 @@ namespace mp {
 int set_error(int code, const char* fmt, ...);  // stores the message, returns code
 void count_launch(int n = 1);
 int check_device();  // MP_OK if the current device is compute capability 10.x
+// Device address (on the current device) of the status word that the GEMM kernels set when a
+// bounded wait expires; defined beside those kernels.
+int gemm_status_device_ptr(int** out);
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 

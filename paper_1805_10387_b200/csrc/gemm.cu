@@ -30,6 +30,8 @@
 #include <cudaTypedefs.h>
 #include <cuda_fp16.h>
 
+#include <mutex>
+
 #include "common.h"
 #include "ptx.cuh"
 
@@ -51,7 +53,7 @@ constexpr int THREADS_FUSED = 64 + 32 * 8;
 constexpr int TMEM_COLS = 512;
 constexpr int STAGING_BYTES = 8 * 32 * 64 * 2;  // epilogue staging: 8 slots of 32 rows x 64 FP16 columns
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + STAGING_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
-constexpr int kModelSMs = 148;                 // used by the split heuristic only
+constexpr int kFallbackSMs = 148;              // split heuristic when no device can be asked
 
 __device__ int g_gemm_status = 0;              // first device-side error (bounded wait expired)
 
@@ -77,6 +79,9 @@ struct GemmParams {
   float* ws;            // FP32 partials [problem][splits][Mo][ws_ld]
   int64_t ws_ld;
   int* flag;            // found_inf word, or null
+  int* status;          // status word of the caller's state object, or null
+  uint64_t wait_ns;     // limit of every wait on a pipeline barrier
+  int no_loads;         // error-path self-test only: the producer issues no load at all
   // Optional fused epilogue (FP16 output only).  Forward flavour: add bias[col] to the FP32 sum,
   // then the activation.  Data-gradient flavour: zero the output where the layer input
   // mask[row, col] (the previous layer's activated FP16 output) is outside the activation's
@@ -101,10 +106,14 @@ __device__ __forceinline__ uint32_t pair_nonfinite(uint32_t w) {
   return __vcmpeq2(w & 0x7C007C00u, 0x7C007C00u);
 }
 
+// A bounded wait ran out: the CTA stops taking work.  The error is recorded in the device-wide
+// status word (which the update and loss-scale kernels consult before they touch the training
+// state) and, when the call was given a state object, in that state's status field.
 template <class B>
-__device__ __forceinline__ void report_timeout(B* bars) {
+__device__ __forceinline__ void report_timeout(B* bars, const GemmParams& p) {
   bars->abort = 1;
   atomicCAS(&g_gemm_status, 0, (int)MP_ERR_TIMEOUT);
+  if (p.status != nullptr) atomicCAS(p.status, 0, (int)MP_ERR_TIMEOUT);
 }
 
 // Row-tile and column-tile index of tile number `tile`.  Consecutive tiles run at the same time
@@ -417,7 +426,8 @@ mp_gemm_kernel(const __grid_constant__ GroupMaps maps, const GemmParams p) {
     uint32_t phase = 0;
     int issued = 0;
     bool ok = true;
-    for (int w = blockIdx.x; w < total_work && ok; w += gridDim.x) {
+    // (no_loads: the error-path self-test; nothing is issued, so nothing is in flight at exit)
+    for (int w = blockIdx.x; w < total_work && ok && !p.no_loads; w += gridDim.x) {
       const int prob = w / p.work_per_problem, wl = w - prob * p.work_per_problem;
       const int split = wl % p.splits, tile = wl / p.splits;
       const CUtensorMap* map_a = &maps.a[prob];
@@ -427,7 +437,7 @@ mp_gemm_kernel(const __grid_constant__ GroupMaps maps, const GemmParams p) {
       const int kb0 = (int)((int64_t)split * p.num_kb / p.splits);
       const int kb1 = (int)((int64_t)(split + 1) * p.num_kb / p.splits);
       for (int kb = kb0; kb < kb1; ++kb) {
-        if (!ptx::mbar_wait(&bars->empty[stage], phase ^ 1)) { ok = false; break; }
+        if (!ptx::mbar_wait(&bars->empty[stage], phase ^ 1, p.wait_ns)) { ok = false; break; }
         if (lane == 0) {
           uint8_t* sA = smem + stage * STAGE_BYTES;
           uint8_t* sB = sA + A_BYTES;
@@ -454,14 +464,14 @@ mp_gemm_kernel(const __grid_constant__ GroupMaps maps, const GemmParams p) {
         if (++stage == STAGES) { stage = 0; phase ^= 1; }
       }
     }
-    if (!ok) report_timeout(bars);
+    if (!ok) report_timeout(bars, p);
     if (!ok || bars->abort) {
       // Leaving early: wait (bounded) until the loads already issued have landed, so that no
       // copy is in flight into this CTA's shared memory when it exits.
       const int pending = issued < STAGES ? issued : STAGES;
       for (int i = 0; i < pending; ++i) {
         if (--stage < 0) { stage = STAGES - 1; phase ^= 1; }
-        ptx::mbar_wait(&bars->full[stage], phase);
+        ptx::mbar_wait(&bars->full[stage], phase, p.wait_ns);
       }
     }
   } else if (warp == 1) {
@@ -479,11 +489,11 @@ mp_gemm_kernel(const __grid_constant__ GroupMaps maps, const GemmParams p) {
       const int kb1 = (int)((int64_t)(split + 1) * p.num_kb / p.splits);
       const int acc = iter & 1;
       const uint32_t acc_phase = (iter >> 1) & 1;
-      if (!ptx::mbar_wait(&bars->tmem_empty[acc], acc_phase ^ 1)) { ok = false; break; }
+      if (!ptx::mbar_wait(&bars->tmem_empty[acc], acc_phase ^ 1, p.wait_ns)) { ok = false; break; }
       ptx::tc_fence_after_sync();
       const uint32_t d_tmem = tmem_base + acc * BN;
       for (int kb = kb0; kb < kb1; ++kb) {
-        if (!ptx::mbar_wait(&bars->full[stage], phase)) { ok = false; break; }
+        if (!ptx::mbar_wait(&bars->full[stage], phase, p.wait_ns)) { ok = false; break; }
         ptx::tc_fence_after_sync();
         if (lane == 0) {
           const uint32_t sA = ptx::smem_u32(smem + stage * STAGE_BYTES);
@@ -508,7 +518,7 @@ mp_gemm_kernel(const __grid_constant__ GroupMaps maps, const GemmParams p) {
       if (ok && lane == 0) ptx::mma_commit(&bars->tmem_full[acc]);
       __syncwarp();
     }
-    if (!ok) report_timeout(bars);
+    if (!ok) report_timeout(bars, p);
   } else {
     // ------------------------------------------------------------ epilogue (warps 2..5)
     const int q = warp & 3;                         // TMEM lane quarter this warp may read
@@ -529,7 +539,7 @@ mp_gemm_kernel(const __grid_constant__ GroupMaps maps, const GemmParams p) {
       uint32_t pass_bits[BN / 32];
       const bool masked = p.mask != nullptr && p.act != 0 && p.out_mode != OUT_PARTIAL;
       if (masked) load_pass_bits(p, row, n0, c_begin, c_count, pass_bits);   // runs under the tile's main loop
-      if (!ptx::mbar_wait(&bars->tmem_full[acc], acc_phase)) { ok = false; break; }
+      if (!ptx::mbar_wait(&bars->tmem_full[acc], acc_phase, p.wait_ns)) { ok = false; break; }
       ptx::tc_fence_after_sync();
       const uint32_t bad = epilogue_tile<WIDE>(p, &maps.out[prob], &maps.ws[prob], stage, nslots, stores,
                                          tmem_base + acc * BN + ((uint32_t)(q * 32) << 16), row, n0, split,
@@ -540,7 +550,7 @@ mp_gemm_kernel(const __grid_constant__ GroupMaps maps, const GemmParams p) {
       ptx::tc_fence_before_sync();
       ptx::mbar_arrive(&bars->tmem_empty[acc]);
     }
-    if (!ok) report_timeout(bars);
+    if (!ok) report_timeout(bars, p);
     if (lane == 0) ptx::bulk_wait_group_all();   // this warp's output stores have left shared memory
   }
 
@@ -643,7 +653,7 @@ mp_gemm_pair_kernel(const __grid_constant__ GroupMaps maps, const GemmParams p) 
       const int kb0 = (int)((int64_t)split * p.num_kb / p.splits);
       const int kb1 = (int)((int64_t)(split + 1) * p.num_kb / p.splits);
       for (int kb = kb0; kb < kb1; ++kb) {
-        if (!ptx::mbar_wait(&bars->empty[stage], phase ^ 1)) { ok = false; break; }
+        if (!ptx::mbar_wait(&bars->empty[stage], phase ^ 1, p.wait_ns)) { ok = false; break; }
         if (lane == 0) {
           uint8_t* sA = smem + stage * STAGE2_BYTES;
           uint8_t* sB = sA + HALF_BYTES;
@@ -675,7 +685,7 @@ mp_gemm_pair_kernel(const __grid_constant__ GroupMaps maps, const GemmParams p) 
         if (++stage == STAGES2) { stage = 0; phase ^= 1; }
       }
     }
-    if (!ok) report_timeout(bars);
+    if (!ok) report_timeout(bars, p);
     if (leader && (!ok || bars->abort)) {
       // Leaving early: the leader's "full" barriers count both CTAs' bytes, so waiting on
       // them (bounded) covers every load still in flight into either CTA; the peer cannot
@@ -683,7 +693,7 @@ mp_gemm_pair_kernel(const __grid_constant__ GroupMaps maps, const GemmParams p) 
       const int pending = issued < STAGES2 ? issued : STAGES2;
       for (int i = 0; i < pending; ++i) {
         if (--stage < 0) { stage = STAGES2 - 1; phase ^= 1; }
-        ptx::mbar_wait(&bars->full[stage], phase);
+        ptx::mbar_wait(&bars->full[stage], phase, p.wait_ns);
       }
     }
   } else if (warp == 1) {
@@ -702,11 +712,11 @@ mp_gemm_pair_kernel(const __grid_constant__ GroupMaps maps, const GemmParams p) 
         const int kb1 = (int)((int64_t)(split + 1) * p.num_kb / p.splits);
         const int acc = iter & 1;
         const uint32_t acc_phase = (iter >> 1) & 1;
-        if (!ptx::mbar_wait(&bars->tmem_empty[acc], acc_phase ^ 1)) { ok = false; break; }
+        if (!ptx::mbar_wait(&bars->tmem_empty[acc], acc_phase ^ 1, p.wait_ns)) { ok = false; break; }
         ptx::tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + acc * BN;
         for (int kb = kb0; kb < kb1; ++kb) {
-          if (!ptx::mbar_wait(&bars->full[stage], phase)) { ok = false; break; }
+          if (!ptx::mbar_wait(&bars->full[stage], phase, p.wait_ns)) { ok = false; break; }
           ptx::tc_fence_after_sync();
           if (lane == 0) {
             const uint32_t sA = ptx::smem_u32(smem + stage * STAGE2_BYTES);
@@ -727,7 +737,7 @@ mp_gemm_pair_kernel(const __grid_constant__ GroupMaps maps, const GemmParams p) 
         if (ok && lane == 0) ptx::mma_commit_pair(&bars->tmem_full[acc], 3);
         __syncwarp();
       }
-      if (!ok) report_timeout(bars);
+      if (!ok) report_timeout(bars, p);
     }
   } else {
     // ------------------------------------------------------------ epilogue (both CTAs)
@@ -749,7 +759,7 @@ mp_gemm_pair_kernel(const __grid_constant__ GroupMaps maps, const GemmParams p) 
       uint32_t pass_bits[BN / 32];
       const bool masked = p.mask != nullptr && p.act != 0 && p.out_mode != OUT_PARTIAL;
       if (masked) load_pass_bits(p, row, n0, c_begin, c_count, pass_bits);   // runs under the tile's main loop
-      if (!ptx::mbar_wait(&bars->tmem_full[acc], acc_phase)) { ok = false; break; }
+      if (!ptx::mbar_wait(&bars->tmem_full[acc], acc_phase, p.wait_ns)) { ok = false; break; }
       ptx::tc_fence_after_sync();
       const uint32_t bad =
           epilogue_tile<WIDE>(p, &maps.out[prob], &maps.ws[prob], stage, nslots, stores,
@@ -763,7 +773,7 @@ mp_gemm_pair_kernel(const __grid_constant__ GroupMaps maps, const GemmParams p) 
       if (lane == 0)
         ptx::mbar_arrive_cluster(ptx::map_to_cta(ptx::smem_u32(&bars->tmem_empty[acc]), 0));
     }
-    if (!ok) report_timeout(bars);
+    if (!ok) report_timeout(bars, p);
     if (lane == 0) ptx::bulk_wait_group_all();   // this warp's output stores have left shared memory
   }
 
@@ -832,9 +842,14 @@ mp_splitk_reduce_kernel(const float* __restrict__ ws, int splits, int Mo, int No
 }
 
 // ------------------------------------------------------------------ host side
+// One-time set-up per device and per kernel flavour (attribute calls, occupancy and symbol
+// queries) is serialised by this mutex, so that first calls from several host threads are safe.
+std::mutex g_setup_mutex;
+
 PFN_cuTensorMapEncodeTiled_v12000 g_encode = nullptr;
 
 int load_encoder() {
+  std::lock_guard<std::mutex> lock(g_setup_mutex);
   if (g_encode) return MP_OK;
   void* fn = nullptr;
   cudaDriverEntryPointQueryResult qres;
@@ -877,6 +892,25 @@ int make_map_ws(CUtensorMap* map, const void* ptr, int64_t ld, int64_t rows, int
   return MP_OK;
 }
 
+// SM count of the current device (the heuristics below size waves with it); kFallbackSMs when no
+// device can be asked, so that a workspace query still answers.
+constexpr int kMaxDevicesCached = 64;
+int model_sms() {
+  static int sms_of[kMaxDevicesCached] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevicesCached) { cudaGetLastError(); return kFallbackSMs; }
+  std::lock_guard<std::mutex> lock(g_setup_mutex);
+  if (sms_of[dev] == 0) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) {
+      cudaGetLastError();
+      return kFallbackSMs;
+    }
+    sms_of[dev] = n;
+  }
+  return sms_of[dev];
+}
+
 // Number of reduction splits: minimise a simple time model (waves of tiles on the SMs plus
 // the workspace round trip).  Depends only on the sizes, so that the workspace query and the
 // launch always agree.
@@ -886,7 +920,8 @@ bool use_pair_kernel(int64_t Mo) { return Mo > 128; }
 int choose_splits(int64_t Mo, int64_t No, int64_t R, int64_t count = 1) {
   const bool pair = use_pair_kernel(Mo);
   const int64_t bm = pair ? 256 : BM;
-  const int64_t slots = pair ? kModelSMs / 2 : kModelSMs;
+  const int sms = model_sms();
+  const int64_t slots = pair ? sms / 2 : sms;
   const int64_t tiles = count * ((Mo + bm - 1) / bm) * ((No + BN - 1) / BN);
   const int64_t num_kb = (R + BK - 1) / BK;
   const double t_kb = 0.42e-6;                   // one 128x256x64 block per SM at ~1.0e13 flop/s
@@ -912,6 +947,8 @@ struct Fuse {
   int64_t ldmask = 0;
   int act = 0;
   float clip = 0.0f;
+  uint64_t wait_ns = ptx::kWaitNs;     // limit of the kernel's barrier waits
+  bool no_loads = false;               // error-path self-test: the producer issues nothing
 };
 
 struct Operand {
@@ -923,7 +960,6 @@ struct Operand {
 
 // The per-kernel set-up below (shared-memory opt-in, cluster occupancy) is a property of the
 // device the call runs on, so it is remembered per device index.
-constexpr int kMaxDevicesCached = 64;
 int current_device_slot() {
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0) dev = 0;
@@ -934,10 +970,13 @@ template <bool A_MN, bool B_MN, bool WIDE>
 int launch(const GroupMaps& maps, const GemmParams& p, int grid, cudaStream_t st) {
   static bool attr_set[kMaxDevicesCached] = {};
   const int slot = current_device_slot();
-  if (!attr_set[slot]) {
-    MP_CUDA_TRY(cudaFuncSetAttribute(mp_gemm_kernel<A_MN, B_MN, WIDE>,
-                                     cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
-    attr_set[slot] = true;
+  {
+    std::lock_guard<std::mutex> lock(g_setup_mutex);
+    if (!attr_set[slot]) {
+      MP_CUDA_TRY(cudaFuncSetAttribute(mp_gemm_kernel<A_MN, B_MN, WIDE>,
+                                       cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
+      attr_set[slot] = true;
+    }
   }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(grid, 1, 1);
@@ -957,12 +996,16 @@ int launch(const GroupMaps& maps, const GemmParams& p, int grid, cudaStream_t st
 template <bool A_MN, bool B_MN, bool WIDE>
 int launch_pair(const GroupMaps& maps, const GemmParams& p, int64_t work, cudaStream_t st) {
   static int max_pairs_of[kMaxDevicesCached] = {};
-  int& max_pairs = max_pairs_of[current_device_slot()];
+  std::unique_lock<std::mutex> lock(g_setup_mutex);
+  int max_pairs = max_pairs_of[current_device_slot()];
   if (max_pairs == 0) {
     MP_CUDA_TRY(cudaFuncSetAttribute(mp_gemm_pair_kernel<A_MN, B_MN, WIDE>,
                                      cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM2_BYTES));
+    int sms = 0, dev = 0;
+    MP_CUDA_TRY(cudaGetDevice(&dev));
+    MP_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(2 * kModelSMs, 1, 1);
+    cfg.gridDim = dim3(2 * sms, 1, 1);
     cfg.blockDim = dim3(WIDE ? THREADS_FUSED : THREADS_PLAIN, 1, 1);
     cfg.dynamicSmemBytes = SMEM2_BYTES;
     cudaLaunchAttribute attr;
@@ -973,8 +1016,9 @@ int launch_pair(const GroupMaps& maps, const GemmParams& p, int64_t work, cudaSt
     int n = 0;
     MP_CUDA_TRY(cudaOccupancyMaxActiveClusters(&n, mp_gemm_pair_kernel<A_MN, B_MN, WIDE>, &cfg));
     if (n < 1) return mp::set_error(MP_ERR_CUDA, "no CTA pair of the GEMM kernel fits on this device");
-    max_pairs = n;
+    max_pairs = max_pairs_of[current_device_slot()] = n;
   }
+  lock.unlock();
   const int pairs = (int)(work < max_pairs ? work : max_pairs);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(2 * pairs, 1, 1);
@@ -992,9 +1036,13 @@ int launch_pair(const GroupMaps& maps, const GemmParams& p, int64_t work, cudaSt
 }
 
 // `count` products of one shape and one set of layouts (operands As[i], Bs[i], outputs outs[i]).
+// dstate: the caller's device state or null; its status word receives device-side errors and, when
+// want_flag is set, its found_inf word the inspection of what is stored.
 int run_gemm(const char* name, int count, const Operand* As, const Operand* Bs, void* const* outs,
-             int64_t ldo, int* flag, bool want_flag, void* workspace, size_t ws_bytes, cudaStream_t st,
+             int64_t ldo, mp_dev_state* dstate, bool want_flag, void* workspace, size_t ws_bytes, cudaStream_t st,
              const Fuse& fuse = Fuse()) {
+  int* flag = dstate ? &dstate->h.found_inf : nullptr;
+  want_flag = want_flag && flag != nullptr;
   if (count < 1 || count > MAX_GROUP)
     return mp::set_error(MP_ERR_INVALID_ARG, "%s: between 1 and %d problems per call", name, MAX_GROUP);
   const Operand& A = As[0];
@@ -1032,7 +1080,7 @@ int run_gemm(const char* name, int count, const Operand* As, const Operand* Bs, 
   const bool fused = has_bias || fuse.act != 0;
   if (fuse.mask != nullptr && count != 1)
     return mp::set_error(MP_ERR_INVALID_ARG, "%s: the masked data gradient takes one problem per call", name);
-  p.splits = fused ? 1 : choose_splits(Mo, No, R, count);   // the fused epilogue needs the whole sum
+  p.splits = (fused || fuse.no_loads) ? 1 : choose_splits(Mo, No, R, count);   // the fused epilogue needs the whole sum
   p.work_per_problem = p.m_tiles * p.n_tiles * p.splits;
   for (int i = 0; i < MAX_GROUP; ++i)
     p.bias[i] = (const uint16_t*)(fuse.biases ? fuse.biases[i < count ? i : 0] : fuse.bias);
@@ -1042,6 +1090,11 @@ int run_gemm(const char* name, int count, const Operand* As, const Operand* Bs, 
   p.ldo = ldo;
   p.ws = (float*)workspace; p.ws_ld = ws_ld_for(No);
   p.flag = flag;
+  p.status = dstate ? &dstate->h.status : nullptr;
+  p.wait_ns = fuse.wait_ns;
+  p.no_loads = fuse.no_loads ? 1 : 0;
+  if (fuse.no_loads && (pair || p.splits != 1 || count != 1 || p.m_tiles * p.n_tiles != 1))
+    return mp::set_error(MP_ERR_INVALID_ARG, "%s: the error-path self-test takes one tile of at most 128 x 256", name);
   p.out_mode = p.splits > 1 ? OUT_PARTIAL : (want_flag ? OUT_F16_FLAG : OUT_F16);
   const size_t ws_floats_per_problem = (size_t)p.splits * (size_t)Mo * (size_t)p.ws_ld;
   if (p.splits > 1) {
@@ -1124,10 +1177,10 @@ int run_gemm(const char* name, int count, const Operand* As, const Operand* Bs, 
 }
 
 // One product: the common case.
-int run_gemm(const char* name, const Operand& A, const Operand& B, void* out, int64_t ldo, int* flag,
+int run_gemm(const char* name, const Operand& A, const Operand& B, void* out, int64_t ldo, mp_dev_state* dstate,
              bool want_flag, void* workspace, size_t ws_bytes, cudaStream_t st, const Fuse& fuse = Fuse()) {
   void* outs[1] = {out};
-  return run_gemm(name, 1, &A, &B, outs, ldo, flag, want_flag, workspace, ws_bytes, st, fuse);
+  return run_gemm(name, 1, &A, &B, outs, ldo, dstate, want_flag, workspace, ws_bytes, st, fuse);
 }
 
 // Output rows, output columns and reduction length of a layer's product `op`.
@@ -1140,6 +1193,24 @@ bool product_dims(int64_t M, int64_t K, int64_t N, int op, int64_t* Mo, int64_t*
 }
 
 }  // namespace
+
+// Device address, on the current device, of the device-wide status word that the GEMM kernels
+// write when a bounded wait runs out.  The update and loss-scale kernels read it.
+int mp::gemm_status_device_ptr(int** out) {
+  static int* addr_of[kMaxDevicesCached] = {};
+  int dev = 0;
+  MP_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevicesCached)
+    return mp::set_error(MP_ERR_INVALID_ARG, "device index %d is outside 0..%d", dev, kMaxDevicesCached - 1);
+  std::lock_guard<std::mutex> lock(g_setup_mutex);
+  if (addr_of[dev] == nullptr) {
+    int* ptr = nullptr;
+    MP_CUDA_TRY(cudaGetSymbolAddress((void**)&ptr, g_gemm_status));
+    addr_of[dev] = ptr;
+  }
+  *out = addr_of[dev];
+  return MP_OK;
+}
 
 extern "C" {
 
@@ -1188,8 +1259,7 @@ int mp_linear_bwd_wgrad_grouped(int count, const void* const* X16, int64_t ldx, 
     return mp::set_error(MP_ERR_INVALID_ARG, "mp_linear_bwd_wgrad_grouped: 1..%d problems, non-null arrays", MAX_GROUP);
   Operand A[MAX_GROUP], B[MAX_GROUP];
   for (int i = 0; i < count; ++i) { A[i] = Operand{X16[i], ldx, true, K, M}; B[i] = Operand{dY16[i], lddy, true, N, M}; }
-  int* flag = state ? &state->dev->h.found_inf : nullptr;
-  return run_gemm("mp_linear_bwd_wgrad_grouped", count, A, B, dW16, lddw, flag, state != nullptr, workspace,
+  return run_gemm("mp_linear_bwd_wgrad_grouped", count, A, B, dW16, lddw, state ? state->dev : nullptr, true, workspace,
                   workspace_bytes, (cudaStream_t)stream);
 }
 
@@ -1216,8 +1286,7 @@ int mp_linear_bwd_wgrad(const void* X16, int64_t ldx, const void* dY16, int64_t 
                         mp_state* state, void* workspace, size_t workspace_bytes, void* stream) {
   const Operand A{X16, ldx, true, K, M};
   const Operand B{dY16, lddy, true, N, M};
-  int* flag = state ? &state->dev->h.found_inf : nullptr;
-  return run_gemm("mp_linear_bwd_wgrad", A, B, dW16, lddw, flag, state != nullptr, workspace,
+  return run_gemm("mp_linear_bwd_wgrad", A, B, dW16, lddw, state ? state->dev : nullptr, true, workspace,
                   workspace_bytes, (cudaStream_t)stream);
 }
 
@@ -1226,6 +1295,8 @@ int mp_linear_bwd_wgrad(const void* X16, int64_t ldx, const void* dY16, int64_t 
 // fixed-size device array: every GPU that loads this library reserves it until the process
 // exits, and every call on that GPU shares it.
 #define MP_STATIC_SCRATCH_FLOATS (8u << 20)   /* 8 Mi floats = 32 MiB */
+static_assert((size_t)MP_STATIC_SCRATCH_FLOATS * sizeof(float) == (size_t)MP_STATIC_SCRATCH_BYTES,
+              "the array and the size the header states must agree");
 static __device__ __align__(256) float g_static_scratch[MP_STATIC_SCRATCH_FLOATS];
 
 namespace {
@@ -1240,6 +1311,7 @@ int static_scratch_for_current_device(float** out) {
   MP_CUDA_TRY(cudaGetDevice(&dev));
   if (dev < 0 || dev >= kMaxDevices)
     return mp::set_error(MP_ERR_INVALID_ARG, "device index %d is outside 0..%d", dev, kMaxDevices - 1);
+  std::lock_guard<std::mutex> lock(g_setup_mutex);
   if (g_static_scratch_addr[dev] == nullptr) {
     float* ptr = nullptr;
     const cudaError_t e = cudaGetSymbolAddress((void**)&ptr, g_static_scratch);
@@ -1267,8 +1339,7 @@ int mp_linear_bwd_wgrad_static(const void* X16, int64_t ldx, const void* dY16, i
   if (int rc = static_scratch_for_current_device(&scratch)) return rc;
   const Operand A{X16, ldx, true, K, M};
   const Operand B{dY16, lddy, true, N, M};
-  int* flag = state ? &state->dev->h.found_inf : nullptr;
-  return run_gemm("mp_linear_bwd_wgrad_static", A, B, dW16, lddw, flag, state != nullptr, scratch,
+  return run_gemm("mp_linear_bwd_wgrad_static", A, B, dW16, lddw, state ? state->dev : nullptr, true, scratch,
                   have, (cudaStream_t)stream);
 }
 
@@ -1325,6 +1396,10 @@ int mp_linear_bwd_dgrad_act(const void* dY16, int64_t lddy, const void* W16, int
   if (act != MP_ACT_NONE) {
     if (!A16) return mp::set_error(MP_ERR_INVALID_ARG, "mp_linear_bwd_dgrad_act: null layer input");
     if (lda < K) return mp::set_error(MP_ERR_INVALID_ARG, "mp_linear_bwd_dgrad_act: lda < K");
+    // the epilogue reads the layer input with 128-bit loads
+    if (!mp::aligned16(A16) || (lda & 7))
+      return mp::set_error(MP_ERR_ALIGNMENT, "mp_linear_bwd_dgrad_act: the layer input must be 16-byte "
+                                             "aligned and lda a multiple of 8");
   }
   const Operand A{dY16, lddy, false, M, N};
   const Operand B{W16, ldw, false, K, N};
@@ -1332,6 +1407,26 @@ int mp_linear_bwd_dgrad_act(const void* dY16, int64_t lddy, const void* W16, int
   f.mask = act != MP_ACT_NONE ? A16 : nullptr; f.ldmask = lda; f.act = act; f.clip = clip;
   return run_gemm("mp_linear_bwd_dgrad_act", A, B, dX16, lddx, nullptr, false, workspace,
                   workspace_bytes, (cudaStream_t)stream, f);
+}
+
+// Error-path self-test: the forward product's one-CTA kernel on a single tile, with its producer
+// warp told to issue no load.  Nothing is ever in flight; the MMA issuer's wait for operands and
+// the epilogue's wait for the accumulator run out after wait_us, the CTA records MP_ERR_TIMEOUT,
+// releases its tensor memory and returns.  Y16 is not written.
+int mp_selftest_wait_timeout(const void* X16, int64_t ldx, const void* W16, int64_t ldw, void* Y16,
+                             int64_t ldy, int64_t M, int64_t K, int64_t N, int64_t wait_us,
+                             mp_state* state, void* stream) {
+  if (wait_us < 1 || wait_us > 2000000)
+    return mp::set_error(MP_ERR_INVALID_ARG, "mp_selftest_wait_timeout: wait_us must be in 1 .. 2000000");
+  if (M > BM || N > BN)
+    return mp::set_error(MP_ERR_INVALID_ARG, "mp_selftest_wait_timeout: one tile only (M <= %d, N <= %d)", BM, BN);
+  const Operand A{X16, ldx, false, M, K};
+  const Operand B{W16, ldw, true, N, K};
+  Fuse f;
+  f.wait_ns = (uint64_t)wait_us * 1000ull;
+  f.no_loads = true;
+  return run_gemm("mp_selftest_wait_timeout", A, B, Y16, ldy, state ? state->dev : nullptr, false, nullptr, 0,
+                  (cudaStream_t)stream, f);
 }
 
 // Synchronises the device and returns the first device-side error recorded by a GEMM kernel

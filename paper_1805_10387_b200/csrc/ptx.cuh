@@ -55,16 +55,17 @@ __device__ __forceinline__ uint64_t globaltimer_ns() {
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
-// Bounded wait: false when the phase did not complete within kWaitNs of wall-clock time
+// Bounded wait: false when the phase did not complete within limit_ns of wall-clock time
 // (measured with the global nanosecond timer, so the bound does not depend on how long a
-// single poll sleeps).  Every legitimate wait in the GEMM pipeline lasts microseconds.
+// single poll sleeps).  Every legitimate wait in the GEMM pipeline lasts microseconds; the
+// library's default limit is kWaitNs.
 constexpr uint64_t kWaitNs = 2000000000ull;   // 2 s
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint64_t limit_ns) {
   if (mbar_try_wait(bar, parity)) return true;
   const uint64_t start = globaltimer_ns();
   for (;;) {
     if (mbar_try_wait(bar, parity)) return true;
-    if (globaltimer_ns() - start > kWaitNs) return false;
+    if (globaltimer_ns() - start > limit_ns) return false;
   }
 }
 
@@ -241,7 +242,9 @@ __device__ __forceinline__ void mma_f16_ss_pair(uint32_t d_tmem, uint64_t a_desc
       : "memory");
 }
 // Arrives on the barrier at this shared-memory offset in every CTA of `cta_mask` once all MMAs
-// issued so far by this thread have completed.
+// issued so far by this thread have completed.  This is an mbarrier arrive delivered to both
+// CTAs of the pair on this GPU; it moves no data.  Every TMA load in this library is a plain
+// per-CTA load from this GPU's own memory.
 __device__ __forceinline__ void mma_commit_pair(uint64_t* bar, uint16_t cta_mask) {
   asm volatile(
       "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64"

@@ -13,7 +13,10 @@
 #include <string.h>
 
 #include <atomic>
+#include <map>
+#include <mutex>
 #include <new>
+#include <utility>
 #include <vector>
 
 #include "common.h"
@@ -187,8 +190,12 @@ __device__ __forceinline__ void update_vec8(const TensorRec& T, int64_t i, const
 template <int KIND>
 __global__ void __launch_bounds__(kThreads)
 mp_master_update_kernel(const TensorRec* __restrict__ tensors, const ChunkRec* __restrict__ chunks,
-                        int64_t n_chunks, mp_dev_state* __restrict__ st, OptArgs o) {
+                        int64_t n_chunks, mp_dev_state* __restrict__ st, OptArgs o,
+                        const int* __restrict__ gemm_status) {
   if (*reinterpret_cast<const volatile int32_t*>(&st->h.found_inf) != 0) return;
+  // a product kernel of this step gave up on a wait: its output is incomplete, apply nothing
+  if (*reinterpret_cast<const volatile int32_t*>(&st->h.status) != 0 ||
+      *reinterpret_cast<const volatile int*>(gemm_status) != 0) return;
   __shared__ Coef s_coef;
   __shared__ unsigned int s_ticket;
   if (threadIdx.x == 0) {
@@ -421,8 +428,13 @@ mp_bias_grad_final_kernel(const float* __restrict__ partial, int slabs, int64_t 
 }
 
 // Loss-scale state machine, one thread (Section 3.1, item 1).
-__global__ void mp_loss_scale_update_kernel(mp_dev_state* st) {
+__global__ void mp_loss_scale_update_kernel(mp_dev_state* st, const int* gemm_status) {
   mp_state_host& h = st->h;
+  // A device-side error freezes the training state: the update above wrote nothing, and the
+  // scale, the counters, the flag and the log stay as they are until the host has read the
+  // status and cleared it.
+  if (h.status == 0 && *gemm_status != 0) h.status = *gemm_status;
+  if (h.status != 0) return;
   mp_log_record rec;
   rec.step = h.step;
   rec.scale_before = h.scale;
@@ -453,17 +465,31 @@ __global__ void mp_loss_scale_update_kernel(mp_dev_state* st) {
   st->log_count += 1;
 }
 
-// Blocks of `kernel` that fit on one SM at once (cached per kernel).  Persistent grids are sized
-// to exactly one resident wave: a grid of more blocks than fit runs in rounds of unequal length.
+// One-word moves between the device state's overflow flag and a caller-owned device word.
+__global__ void mp_flag_export_kernel(const mp_dev_state* st, int32_t* word) {
+  *word = st->h.found_inf != 0 ? 1 : 0;
+}
+__global__ void mp_flag_import_kernel(mp_dev_state* st, const int32_t* word) {
+  if (*word != 0) st->h.found_inf = 1;
+}
+
+// Blocks of `kernel` that fit on one SM at once, remembered per (device, kernel).  Persistent
+// grids are sized to exactly one resident wave: a grid of more blocks than fit runs in rounds
+// of unequal length.
 template <class K>
 int resident_blocks_per_sm(K kernel) {
-  static int cached = 0;
-  if (cached == 0) {
-    int n = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, kThreads, 0) != cudaSuccess || n < 1) n = 1;
-    cached = n;
-  }
-  return cached;
+  static std::mutex mu;
+  static std::map<std::pair<int, const void*>, int> cache;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) dev = 0;
+  const std::pair<int, const void*> key(dev, reinterpret_cast<const void*>(kernel));
+  std::lock_guard<std::mutex> lock(mu);
+  auto it = cache.find(key);
+  if (it != cache.end()) return it->second;
+  int n = 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, kThreads, 0) != cudaSuccess || n < 1) n = 1;
+  cache[key] = n;
+  return n;
 }
 
 int grid_for(int64_t work_blocks, int sm_count, int per_sm) {
@@ -560,6 +586,28 @@ int mp_state_read_log(mp_state* s, mp_log_record* out, int max_records, int* n_o
   return MP_OK;
 }
 
+int mp_state_export_flag(const mp_state* s, int32_t* word, void* stream) {
+  if (!s || !word) return mp::set_error(MP_ERR_INVALID_ARG, "mp_state_export_flag: null argument");
+  if (reinterpret_cast<uintptr_t>(word) & 3u)
+    return mp::set_error(MP_ERR_ALIGNMENT, "mp_state_export_flag: word must be 4-byte aligned");
+  if (int rc = mp::check_device()) return rc;
+  mp_flag_export_kernel<<<1, 1, 0, (cudaStream_t)stream>>>(s->dev, word);
+  mp::count_launch();
+  MP_CUDA_TRY(cudaGetLastError());
+  return MP_OK;
+}
+
+int mp_state_import_flag(mp_state* s, const int32_t* word, void* stream) {
+  if (!s || !word) return mp::set_error(MP_ERR_INVALID_ARG, "mp_state_import_flag: null argument");
+  if (reinterpret_cast<uintptr_t>(word) & 3u)
+    return mp::set_error(MP_ERR_ALIGNMENT, "mp_state_import_flag: word must be 4-byte aligned");
+  if (int rc = mp::check_device()) return rc;
+  mp_flag_import_kernel<<<1, 1, 0, (cudaStream_t)stream>>>(s->dev, word);
+  mp::count_launch();
+  MP_CUDA_TRY(cudaGetLastError());
+  return MP_OK;
+}
+
 int mp_update_plan_create(int n, void* const* g16, void* const* w32, void* const* m,
                           void* const* v, void* const* w16, const int64_t* count,
                           mp_update_plan** out) {
@@ -635,6 +683,8 @@ int mp_master_update(mp_update_plan* plan, mp_state* state, const mp_optim_confi
   if (int rc = mp::check_device()) return rc;
   if (plan->n_chunks == 0) return MP_OK;
   cudaStream_t st = (cudaStream_t)stream;
+  int* gemm_status = nullptr;
+  if (int rc = mp::gemm_status_device_ptr(&gemm_status)) return rc;
   const OptArgs o{opt->lr, opt->beta1, opt->beta2, opt->eps, opt->momentum, opt->weight_decay};
   if (check_mode == 1) {
     // (the 2 B/element inspection, unlike the update, is faster as one resident wave)
@@ -648,10 +698,10 @@ int mp_master_update(mp_update_plan* plan, mp_state* state, const mp_optim_confi
   const int grid = grid_for(plan->n_chunks, plan->sm_count, per_sm);
   if (opt->kind == MP_OPT_ADAM)
     mp_master_update_kernel<MP_OPT_ADAM><<<grid, kThreads, 0, st>>>(
-        plan->d_tensors, plan->d_chunks, plan->n_chunks, state->dev, o);
+        plan->d_tensors, plan->d_chunks, plan->n_chunks, state->dev, o, gemm_status);
   else
     mp_master_update_kernel<MP_OPT_MOMENTUM><<<grid, kThreads, 0, st>>>(
-        plan->d_tensors, plan->d_chunks, plan->n_chunks, state->dev, o);
+        plan->d_tensors, plan->d_chunks, plan->n_chunks, state->dev, o, gemm_status);
   mp::count_launch();
   MP_CUDA_TRY(cudaGetLastError());
   return MP_OK;
@@ -660,7 +710,9 @@ int mp_master_update(mp_update_plan* plan, mp_state* state, const mp_optim_confi
 int mp_loss_scale_update(mp_state* state, void* stream) {
   if (!state) return mp::set_error(MP_ERR_INVALID_ARG, "mp_loss_scale_update: null state");
   if (int rc = mp::check_device()) return rc;
-  mp_loss_scale_update_kernel<<<1, 1, 0, (cudaStream_t)stream>>>(state->dev);
+  int* gemm_status = nullptr;
+  if (int rc = mp::gemm_status_device_ptr(&gemm_status)) return rc;
+  mp_loss_scale_update_kernel<<<1, 1, 0, (cudaStream_t)stream>>>(state->dev, gemm_status);
   mp::count_launch();
   MP_CUDA_TRY(cudaGetLastError());
   return MP_OK;
@@ -696,7 +748,9 @@ static int bias_vecs(int64_t N) {        // 16-byte vectors per row and warp, as
 
 static int bias_slabs(int64_t M, int64_t N) {
   const int64_t col_blocks = (N + kBiasCols - 1) / kBiasCols;
-  int64_t want = 8 * 148 / col_blocks;
+  int sms = 0;
+  if (sm_count_of_current_device(&sms) != MP_OK || sms < 1) sms = 148;   // no device to ask: a B200's count
+  int64_t want = 8 * (int64_t)sms / col_blocks;
   const int64_t rows_per_pass = 32 * (32 / bias_vecs(N));     // rows one block reads at once
   const int64_t by_rows = (M + rows_per_pass - 1) / rows_per_pass;
   if (want > by_rows) want = by_rows;

@@ -84,10 +84,13 @@ SIGNATURES = {
     "mp_state_destroy": (_i32, [_p]),
     "mp_state_read": (_i32, [_p, C.POINTER(StateHost), _p]),
     "mp_state_write": (_i32, [_p, C.POINTER(StateHost), _p]),
+    "mp_state_export_flag": (_i32, [_p, _p, _p]),
+    "mp_state_import_flag": (_i32, [_p, _p, _p]),
     "mp_state_read_log": (_i32, [_p, C.POINTER(LogRecord), _i32, C.POINTER(_i32), _p]),
     "mp_update_plan_create": (_i32, [_i32, C.POINTER(_p), C.POINTER(_p), C.POINTER(_p),
                                      C.POINTER(_p), C.POINTER(_p), C.POINTER(_i64), C.POINTER(_p)]),
     "mp_update_plan_destroy": (_i32, [_p]),
+    "mp_selftest_wait_timeout": (_i32, [_p, _i64, _p, _i64, _p, _i64, _i64, _i64, _i64, _i64, _p, _p]),
     "mp_gemm_device_status": (_i32, [C.POINTER(_i32)]),
     "mp_last_error": (C.c_char_p, []),
     "mp_kernel_launch_count": (_i64, []),
@@ -322,6 +325,26 @@ def mp_scale_upstream(g32, dY16, state):
 def mp_check_finite(g16, state):
     assert g16.is_contiguous()
     _check(lib().mp_check_finite(_dev(g16, torch.float16), g16.numel(), state.handle, _stream()))
+
+
+def mp_state_export_flag(state, word):
+    """word[0] (int32 CUDA tensor) = the state's overflow flag, on the stream."""
+    _check(lib().mp_state_export_flag(state.handle, _dev(word, torch.int32), _stream()))
+
+
+def mp_state_import_flag(state, word):
+    """ORs word[0] != 0 (int32 CUDA tensor) into the state's overflow flag, on the stream."""
+    _check(lib().mp_state_import_flag(state.handle, _dev(word, torch.int32), _stream()))
+
+
+def mp_selftest_wait_timeout(X16, W16, Y16, wait_us: int, state=None):
+    """Error-path self-test: one tile of the forward kernel whose loader fetches nothing, so its
+    bounded waits run out after wait_us microseconds and it reports MP_ERR_TIMEOUT."""
+    (x, ldx), (w, ldw), (y, ldy) = _mat(X16), _mat(W16), _mat(Y16)
+    M, K = X16.shape
+    N = W16.shape[1]
+    _check(lib().mp_selftest_wait_timeout(x, ldx, w, ldw, y, ldy, M, K, N, int(wait_us),
+                                          state.handle if state is not None else None, _stream()))
 
 
 def mp_gemm_device_status() -> int:

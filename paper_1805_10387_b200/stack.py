@@ -13,7 +13,7 @@ from __future__ import annotations
 
 import torch
 
-from . import mp
+from . import dp, mp
 
 
 def _align(n: int, a: int = 8) -> int:
@@ -24,13 +24,18 @@ class LinearStack:
     def __init__(self, shapes, chained, optimizer="adam", lr=1e-3, beta1=0.9, beta2=0.999,
                  eps=1e-8, momentum=0.9, weight_decay=0.0, init_scale=65536.0,
                  growth_interval=1000, min_scale=1.0, max_scale=2.0 ** 24, dynamic=True,
-                 device="cuda", acts=None, clip=20.0, bias=False, overflow_tolerance=1, lstm=None):
+                 device="cuda", acts=None, clip=20.0, bias=False, overflow_tolerance=1, lstm=None,
+                 comm=None, shard_update=False):
         """acts[l]: mp.MP_ACT_* after layer l's product (a layer whose output feeds no chained
         layer must have MP_ACT_NONE); bias: every layer gets a bias vector; lstm[l]: layer l's
         product is the gate pre-activation of an LSTM cell (N = 4 H, gate order i, f, g, o): the
         cell kernels turn it and the cell state c_prev[l] into c_new[l] and h[l], the gradient
         entering the layer is that of h ([M, H]), and the cell's backward kernel produces the
-        gate gradient that the layer's two backward products consume."""
+        gate gradient that the layer's two backward products consume.
+        comm: data-parallel exchange (an object with the methods of dp.Comm; None = one rank).
+        shard_update: with a comm of G ranks, each rank keeps and updates only its 1/G slice of
+        the FP32 master and moments (reduce-scatter of the gradients before, all-gather of the
+        FP16 weights after) instead of every rank repeating the whole update."""
         self.shapes = [tuple(s) for s in shapes]
         self.chained = list(chained)
         self.L = len(shapes)
@@ -62,28 +67,51 @@ class LinearStack:
         for _, _, n in self.shapes:
             boffs.append(total)
             total += _align(n) if self.has_bias else 0
-        self.offsets, self.total = offs, total
+        self.comm = comm
+        self.world = comm.world if comm is not None else 1
+        self.rank = comm.rank if comm is not None else 0
+        self.shard_update = bool(shard_update) and self.world > 1
+        if self.shard_update:
+            # equal slices that start on 16-byte boundaries: pad the flat range to 8 * world elements
+            total = dp.padded_total(total, self.world)
+        self.offsets, self.boffsets, self.sizes, self.total = offs, boffs, sizes, total
         f16 = dict(dtype=torch.float16, device=self.device)
         f32 = dict(dtype=torch.float32, device=self.device)
         self.w16_flat = torch.zeros(total, **f16)
         self.dw_flat = torch.zeros(total, **f16)
-        self.w32_flat = torch.zeros(total, **f32)
-        self.m_flat = torch.zeros(total, **f32)
-        self.v_flat = torch.zeros(total, **f32) if optimizer == "adam" else None
         view = lambda flat, l: flat[offs[l]:offs[l] + sizes[l]].view(self.shapes[l][1], self.ldw[l])
+        bview = lambda flat, l: flat[boffs[l]:boffs[l] + self.shapes[l][2]] if self.has_bias else None
         self.w16 = [view(self.w16_flat, l) for l in range(self.L)]
         self.dw = [view(self.dw_flat, l) for l in range(self.L)]
-        self.w32 = [view(self.w32_flat, l) for l in range(self.L)]
-        self.m = [view(self.m_flat, l) for l in range(self.L)]
-        self.v = [view(self.v_flat, l) for l in range(self.L)] if self.v_flat is not None else None
-        bview = lambda flat, l: flat[boffs[l]:boffs[l] + self.shapes[l][2]] if self.has_bias else None
         self.b16 = [bview(self.w16_flat, l) for l in range(self.L)]
         self.db = [bview(self.dw_flat, l) for l in range(self.L)]
-        self.b32 = [bview(self.w32_flat, l) for l in range(self.L)]
-        # one plan over the whole flat range: padding columns hold zeros and stay zero
-        self.plan = mp.UpdatePlan([self.dw_flat], [self.w32_flat], [self.m_flat],
-                                  [self.v_flat] if self.v_flat is not None else None,
-                                  [self.w16_flat])
+        if not self.shard_update:
+            self.shard = (0, total)
+            self.w32_flat = torch.zeros(total, **f32)
+            self.m_flat = torch.zeros(total, **f32)
+            self.v_flat = torch.zeros(total, **f32) if optimizer == "adam" else None
+            self.w32 = [view(self.w32_flat, l) for l in range(self.L)]
+            self.m = [view(self.m_flat, l) for l in range(self.L)]
+            self.v = [view(self.v_flat, l) for l in range(self.L)] if self.v_flat is not None else None
+            self.b32 = [bview(self.w32_flat, l) for l in range(self.L)]
+            # one plan over the whole flat range: padding columns hold zeros and stay zero
+            self.plan = mp.UpdatePlan([self.dw_flat], [self.w32_flat], [self.m_flat],
+                                      [self.v_flat] if self.v_flat is not None else None,
+                                      [self.w16_flat])
+        else:
+            # this rank's slice [lo, hi) of the flat parameter range: the only part of the FP32
+            # master and of the moments that exists here
+            lo, hi = self.shard = dp.shard_params(total, self.rank, self.world)
+            n = hi - lo
+            self.w32_flat = torch.zeros(n, **f32)
+            self.m_flat = torch.zeros(n, **f32)
+            self.v_flat = torch.zeros(n, **f32) if optimizer == "adam" else None
+            self.w32 = self.m = self.v = self.b32 = None      # per-layer FP32 views do not exist
+            self.dw_shard = torch.zeros(n, **f16)             # reduced gradients of the slice
+            self.flag_word = torch.zeros(1, dtype=torch.int32, device=self.device)
+            self.plan = mp.UpdatePlan([self.dw_shard], [self.w32_flat], [self.m_flat],
+                                      [self.v_flat] if self.v_flat is not None else None,
+                                      [self.w16_flat[lo:lo + n]])
 
         # activations and their gradients
         self.x = [None] * self.L
@@ -154,11 +182,27 @@ class LinearStack:
     def load_weights(self, l: int, w32: torch.Tensor, w16: torch.Tensor, b32=None, b16=None):
         """Copies an FP32 master [K,N] and its FP16 working copy (and a bias pair) into the stack."""
         n = self.shapes[l][2]
-        self.w32[l][:, :n].copy_(w32)
         self.w16[l][:, :n].copy_(w16)
-        if b32 is not None:
-            self.b32[l].copy_(b32)
+        if b16 is not None:
             self.b16[l].copy_(b16)
+        if not self.shard_update:
+            self.w32[l][:, :n].copy_(w32)
+            if b32 is not None:
+                self.b32[l].copy_(b32)
+            return
+        # sharded master: keep the part of this tensor that falls into the rank's slice
+        lo, hi = self.shard
+
+        def place(dst_off, src_flat):
+            a, b = max(lo, dst_off), min(hi, dst_off + src_flat.numel())
+            if a < b:
+                self.w32_flat[a - lo:b - lo].copy_(src_flat[a - dst_off:b - dst_off])
+        k = self.shapes[l][1]
+        padded = torch.zeros(k, self.ldw[l], dtype=torch.float32, device=self.device)
+        padded[:, :n].copy_(w32)
+        place(self.offsets[l], padded.reshape(-1))
+        if b32 is not None:
+            place(self.boffsets[l], b32.to(self.device, torch.float32).reshape(-1))
 
     def X(self, l): return self.x[l][:, :self.shapes[l][1]]
     def Y(self, l): return self.y[l][:, :self.shapes[l][2]]
@@ -173,7 +217,6 @@ class LinearStack:
 
     # ---- optional per-call device timing (CUDA events on the launching stream) ----
     events = None   # set to a list to collect (name, start_event, end_event)
-    grad_sync = None  # data-parallel runs: callable that all-reduces the flat FP16 gradient
 
     only = None       # set to a set of call classes to make step() issue only those calls
 
@@ -308,6 +351,11 @@ class LinearStack:
         """xs[l]: FP16 [M,K] CUDA tensor (row pitch a multiple of 8) for a layer that is not
         chained; gs[l]: contiguous FP32 [M,N] CUDA tensor, the unscaled gradient entering a layer
         whose output feeds no chained layer."""
+        self.products(xs, gs)
+        self.finish()
+
+    def products(self, xs, gs):
+        """The forward and backward products of the step (arguments as for step())."""
         for l in range(self.L):
             if not self.chained[l]:
                 self.x[l] = xs[l]
@@ -374,11 +422,55 @@ class LinearStack:
                 else:   # the layer below is activated: mask with its stored output (= this layer's input)
                     self._call("dgrad", mp.mp_linear_bwd_dgrad_act, self.dY(l), self.W16(l), X, self.dX(l),
                                below, self.clip, self.workspace)
-        if self.grad_sync is not None and self.only is None:   # data parallel: sum the FP16 gradients over ranks,
-            self.grad_sync(self.dw_flat)     # then inspect the reduced gradients in the update call
-        self._call("update", mp.mp_master_update, self.plan, self.state, self.opt,
-                   0 if self.grad_sync is None else 1)
+
+    def finish(self):
+        """Everything after the backward products: the gradient exchange of a data-parallel run,
+        the fused update and the loss-scale state machine.  The parts are methods of their own
+        so that a test can drive several stacks that stand for ranks in lockstep."""
+        if self.only is not None:
+            self._call("update", mp.mp_master_update, self.plan, self.state, self.opt, 0)
+            self._call("scaler", mp.mp_loss_scale_update, self.state)
+            return
+        self.exchange_gradients()
+        self.inspect_exchanged()
+        self.apply_update()
+        self.publish_weights()
         self._call("scaler", mp.mp_loss_scale_update, self.state)
+
+    def exchange_gradients(self):
+        """Data parallel (Section 4 of the paper): the FP16 weight gradients are summed over the
+        ranks; replicated update: all-reduce of the flat buffer; sharded update: reduce-scatter,
+        each rank receiving the sum of its slice."""
+        if self.comm is None:
+            return
+        if self.shard_update:
+            self.comm.reduce_scatter(self.dw_flat, self.dw_shard)
+        else:
+            self.comm.all_reduce(self.dw_flat)
+
+    def inspect_exchanged(self):
+        """Sharded update only: a rank sees just its slice of the summed gradients, so it
+        inspects that slice and the ranks agree on the flag with a one-word max-reduction.  (The
+        replicated update inspects the whole reduced buffer inside the update call instead; the
+        flags the weight-gradient kernels raised on local gradients stay set either way: an inf
+        in a local gradient is an inf in the sum.)"""
+        if not self.shard_update:
+            return
+        self._call("check", mp.mp_check_finite, self.dw_shard, self.state)
+        mp.mp_state_export_flag(self.state, self.flag_word)
+        self.comm.all_reduce_max(self.flag_word)
+        mp.mp_state_import_flag(self.state, self.flag_word)
+
+    def apply_update(self):
+        # replicated data-parallel update: the call inspects the reduced gradients itself
+        self._call("update", mp.mp_master_update, self.plan, self.state, self.opt,
+                   1 if (self.comm is not None and not self.shard_update) else 0)
+
+    def publish_weights(self):
+        """Sharded update only: every rank rewrote the FP16 copy of its slice; gather the slices."""
+        if self.shard_update:
+            lo, hi = self.shard
+            self.comm.all_gather(self.w16_flat, self.w16_flat[lo:hi])
 
     def close(self):
         self.plan.close()

@@ -54,3 +54,14 @@ def test_argument_errors_need_no_gpu():
     assert L.mp_linear_fwd(p16, 4, p16, 8, p16, 8, 8, 8, 8, None, 0, None) == mp.MP_ERR_INVALID_ARG
     assert L.mp_linear_fwd(p16, 12, p16, 8, p16, 8, 8, 8, 8, None, 0, None) == mp.MP_ERR_ALIGNMENT
     assert L.mp_linear_fwd(p16 + 2, 8, p16, 8, p16, 8, 8, 8, 8, None, 0, None) == mp.MP_ERR_ALIGNMENT
+    # the masked data gradient reads the layer input with 128-bit loads: checked on the host too
+    args = lambda a16, lda: (p16, 8, p16, 8, a16, lda, p16, 8, 8, 8, 8, mp.MP_ACT_RELU, ctypes.c_float(0.0),
+                             None, 0, None)
+    assert L.mp_linear_bwd_dgrad_act(*args(p16 + 2, 8)) == mp.MP_ERR_ALIGNMENT
+    assert L.mp_linear_bwd_dgrad_act(*args(p16, 12)) == mp.MP_ERR_ALIGNMENT
+    assert L.mp_linear_bwd_dgrad_act(*args(p16, 4)) == mp.MP_ERR_INVALID_ARG
+    assert L.mp_linear_bwd_dgrad_act(*args(None, 8)) == mp.MP_ERR_INVALID_ARG
+    # the error-path self-test refuses more than one tile and limits outside 1 us .. 2 s
+    st = lambda M, N, us: L.mp_selftest_wait_timeout(p16, 8, p16, 8, p16, 8, M, 8, N, us, None, None)
+    assert st(8, 8, 0) == mp.MP_ERR_INVALID_ARG and st(8, 8, 3_000_000) == mp.MP_ERR_INVALID_ARG
+    assert st(129, 8, 100) == mp.MP_ERR_INVALID_ARG and st(8, 257, 100) == mp.MP_ERR_INVALID_ARG

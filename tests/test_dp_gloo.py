@@ -82,3 +82,65 @@ def test_two_ranks_reduce_and_agree(plant_inf):
         # sum of the two shard gradients = gradient over all rows, up to FP16 roundings
         a = full[1].view(np.float16).astype(np.float64); b = full[2].view(np.float16).astype(np.float64)
         assert (np.abs(a - b) <= 2.0 ** -9 * np.abs(a) + 1e-3 * np.sqrt((a * a).mean())).all()
+
+
+def test_parameter_slices_are_equal_and_aligned():
+    for total, world in ((64632, 2), (64632, 3), (1, 8), (75_497_472, 8), (12_846_400 + 29 * 8, 7)):
+        padded = dp.padded_total(total, world)
+        assert padded >= total and padded % (8 * world) == 0 and padded - total < 8 * world
+        edges = [dp.shard_params(padded, r, world) for r in range(world)]
+        assert edges[0][0] == 0 and edges[-1][1] == padded
+        assert all(a[1] == b[0] for a, b in zip(edges, edges[1:]))
+        assert len({hi - lo for lo, hi in edges}) == 1
+        assert all(lo % 8 == 0 for lo, _ in edges)              # 16-byte boundaries for FP16 and FP32
+    with pytest.raises(ValueError):
+        dp.shard_params(100, 0, 3)
+
+
+def _shard_worker(rank, world, port, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    comm = dp.Comm()
+    total = dp.padded_total(1000 + 13, world)                   # ragged: the last slice holds padding
+    rng = np.random.default_rng(100 + rank)
+    mine = torch.from_numpy(rng.integers(-8, 9, total).astype(np.float16))   # exact in FP16, any order
+    flat = mine.clone()
+    lo, hi = dp.shard_params(total, rank, world)
+    got = torch.zeros(hi - lo, dtype=torch.float16)
+    comm.reduce_scatter(flat, got)
+    assert torch.equal(flat, mine)                              # the input is left alone
+    # all-gather: every rank contributes (its slice + rank) and ends with the same full buffer
+    full = torch.zeros(total, dtype=torch.float16)
+    full[lo:hi] = got + rank
+    comm.all_gather(full, full[lo:hi])
+    word = torch.tensor([1 if rank == world - 1 else 0], dtype=torch.int32)
+    comm.all_reduce_max(word)
+    out.put((rank, mine.numpy().copy(), got.numpy().copy(), full.numpy().copy(), int(word[0])))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+@pytest.mark.parametrize("world", [2, 3])
+def test_sharded_exchange_bookkeeping(world):
+    """reduce-scatter gives each rank the sum of its slice, all-gather rebuilds the full buffer on
+    every rank, the flag word takes the max: the exchanges of the sharded-update schedule."""
+    ctx = tmp.get_context("spawn")
+    q = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_shard_worker, args=(r, world, port, q)) for r in range(world)]
+    for p in procs:
+        p.start()
+    got = sorted((q.get(timeout=120) for _ in range(world)), key=lambda x: x[0])
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    total = got[0][1].size
+    want_sum = sum(g[1].astype(np.float32) for g in got)
+    want_full = np.empty(total, np.float32)
+    for r, g in enumerate(got):
+        lo, hi = dp.shard_params(total, r, world)
+        assert (g[2].astype(np.float32) == want_sum[lo:hi]).all()
+        want_full[lo:hi] = want_sum[lo:hi] + r
+    for g in got:
+        assert (g[3].astype(np.float32) == want_full).all()
+        assert g[4] == 1

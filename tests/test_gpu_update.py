@@ -87,10 +87,13 @@ def test_check_finite_exhaustive_patterns(orc, mp):
     fin = allbits[want == 0]
     mp.mp_check_finite(_dev16(fin), st)
     assert st.read().found_inf == 0
-    for h in allbits[want == 1][::37]:
-        g = fin[:100].copy(); g[50] = h
-        mp.mp_check_finite(_dev16(g), st)
-        assert st.read().found_inf == 1
+    bad = allbits[want == 1]
+    assert bad.size == 2048                              # 2 infinities + 2046 NaNs
+    buf = torch.from_numpy(fin[:100].view(np.int16).copy()).cuda()
+    for h in bad:                                        # all of them, one at a time
+        buf[50] = int(np.int16(np.uint16(h).view(np.int16)))
+        mp.mp_check_finite(buf.view(torch.float16), st)
+        assert st.read().found_inf == 1, hex(int(h))
         mp.mp_loss_scale_update(st)
     st.close()
 

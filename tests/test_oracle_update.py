@@ -41,6 +41,60 @@ def test_flag_position_sweep(orc):
     assert orc.found_inf(np.empty(0, np.uint16)) == 0
 
 
+# ------------------------------------------------------- upstream scaling
+def _hx(h):
+    return np.array([h], np.uint16)
+
+
+def test_scale_upstream_scales_in_fp32_before_the_one_rounding(orc):
+    """rn16(S * g32): the product is formed in FP32 and rounded to FP16 once.
+
+    Each case has a value fixed by the binary16 format; rounding g to FP16 first, or
+    multiplying in FP16, gives a different one."""
+    one = lambda g, S: int(orc.scale_upstream(np.array([g], np.float32), S)[0])
+    # 2^-26 is below half the smallest subnormal: FP16 holds it as 0, yet 2^16 * 2^-26 = 2^-10 is a normal
+    assert one(2.0 ** -26, 2.0 ** 16) == 0x1400
+    assert one(-(2.0 ** -26), 2.0 ** 16) == 0x9400
+    # g = 1 + 2^-11 is a tie that FP16 rounds to 1.0; with S = 3 the FP32 product 3 + 1.5 * 2^-10 lies above
+    # the midpoint between 3 and 3 + 2^-9, so the result is 3 + 2^-9; rounding g first would give 3.0 = 0x4200
+    assert one(1.0 + 2.0 ** -11, 3.0) == 0x4201
+    # S = 1 reduces to the plain conversion: the fixture's ties and thresholds
+    for line in open(os.path.join(GOLD, "fp16_thresholds.txt")):
+        line = line.split("#")[0].split()
+        if not line:
+            continue
+        g = np.array([int(line[0], 16)], np.uint32).view(np.float32)
+        assert int(orc.scale_upstream(g, 1.0)[0]) == int(line[1], 16), line
+    # overflow of the scaled value: 65520 is the first value that becomes inf
+    assert one(65519.0 / 1024.0, 1024.0) == 0x7BFF          # 65519 < 65520 -> 65504
+    assert one(65520.0 / 1024.0, 1024.0) == 0x7C00
+    assert one(-64.0, 1024.0) == 0xFC00                     # -65536 -> -inf
+    assert one(1.0, 2.0 ** 16) == 0x7C00
+    assert one(np.inf, 2.0) == 0x7C00 and one(-np.inf, 2.0) == 0xFC00
+    nan = one(np.nan, 2.0)
+    assert (nan & 0x7C00) == 0x7C00 and (nan & 0x03FF) != 0
+    assert one(0.0, 2.0 ** 16) == 0x0000 and one(-0.0, 2.0 ** 16) == 0x8000
+    assert orc.scale_upstream(np.empty(0, np.float32), 4.0).size == 0
+
+
+def test_scale_upstream_against_library_product(orc):
+    """10^6 seeded floats, S = 10 (not a power of two) and S = 2^15: numpy's float32 product cast to
+    float16 is the same definition in an independent implementation."""
+    rng = np.random.default_rng(77)
+    g = (rng.standard_normal(1_000_000) * np.exp(rng.uniform(-18, 9, 1_000_000))).astype(np.float32)
+    g[:8] = [0.0, -0.0, np.inf, -np.inf, 6552.0, 6551.9, 2.0 ** -27, -(2.0 ** -24)]
+    for S in (10.0, 2.0 ** 15, 3.0, 1.0):
+        with np.errstate(over="ignore"):
+            want = (np.float32(S) * g).astype(np.float16).view(np.uint16)
+        got = orc.scale_upstream(g, S)
+        assert (got == want).all(), S
+        assert ((got & 0x7C00) == 0x7C00).any() and (got == 0).any()       # both ends exercised
+    # and not the result of rounding first: on this sample the two differ somewhere
+    with np.errstate(over="ignore"):
+        first = (g.astype(np.float16).astype(np.float32) * np.float32(10.0)).astype(np.float16).view(np.uint16)
+    assert (first != orc.scale_upstream(g, 10.0)).any()
+
+
 # ------------------------------------------------------------------ Adam
 ADAM = dict(lr=1e-3, b1=0.9, b2=0.999, eps=1e-8)
 
