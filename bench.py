@@ -36,19 +36,19 @@ if ROOT not in sys.path:
 METRIC = "MP train step: GEMM TFLOP/s and master-update GB/s, % of B200 peak"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
-# DRAM bytes per launch of the GEMM kernel from one ncu capture (dram__bytes_read.sum +
-# dram__bytes_write.sum, mean over one step's product launches; on c2 a launch holds four layers'
-# products, 4 x 95.4 MB algorithmic), keyed by workload, valid only for the kernel source it was
-# taken on.
-NCU_TRAFFIC = {"sha": "735224e192c28da6", "bytes_per_launch": {"c2": 401.4e6}}
+# DRAM bytes per launch of the product kernels from one ncu capture per workload (dram__bytes_read.sum
+# + dram__bytes_write.sum summed over one step's product launches, split-reduction kernels included,
+# divided by their number; on c2 a launch holds four layers' products, 4 x 95.4 MB algorithmic), valid
+# only for the kernel source it was taken on.
+NCU_TRAFFIC = {"sha": "0874106332883409", "bytes_per_launch": {"c2": 402.4e6, "c3": 82.3e6, "c4": 116.2e6}}
 # flop per clock and SM of the FP16 tensor pipe (one 128 x 256 x 16 MMA per SM in 128 clocks)
 TENSOR_FLOP_PER_CLK_SM = 8192
 
 
 # DRAM bytes per parameter of the fused update from one ncu capture at 1e8 parameters in 64 tensors
-# (2.7400 GB per launch); a launch over P parameters moves P times this (traffic grows in
+# (2.7406 GB per launch); a launch over P parameters moves P times this (traffic grows in
 # proportion: every parameter is touched once), valid only for the kernel source it was taken on.
-NCU_UPDATE_TRAFFIC = {"sha": "d29d336f54d27289", "bytes_per_param": 27.40}
+NCU_UPDATE_TRAFFIC = {"sha": "3718ba9d82009239", "bytes_per_param": 27.41}
 
 
 def update_kernel_sha():
@@ -247,7 +247,7 @@ def run_update_sweep(args, sampler=None, steps=None, settle_s=1.0):
         sampler = ClockSampler(int(os.environ.get("LOCAL_RANK", "0")))
         sampler.start()
     windows = []
-    launches0 = mp.mp_kernel_launch_count()
+    timed_launches = 0
     for P, n in ((1_000_000, 1), (10_000_000, 8), (100_000_000, 64), (1_000_000_000, 500)):
         if P > args.max_params:
             break
@@ -277,8 +277,10 @@ def run_update_sweep(args, sampler=None, steps=None, settle_s=1.0):
             mp.mp_loss_scale_update(st)
 
         def timed(mode, reps):
+            nonlocal timed_launches
             settle(lambda: one(mode), settle_s, torch.cuda.synchronize)
             t0 = time.time()
+            n0 = mp.mp_kernel_launch_count()
             ts = []
             for _ in range(reps):
                 a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -288,6 +290,7 @@ def run_update_sweep(args, sampler=None, steps=None, settle_s=1.0):
                 mp.mp_loss_scale_update(st)
                 ts.append((a, b))
             torch.cuda.synchronize()
+            timed_launches += mp.mp_kernel_launch_count() - n0
             if P >= 100_000_000:
                 windows.append((t0, time.time()))
             return sum(a.elapsed_time(b) for a, b in ts) / reps
@@ -318,7 +321,7 @@ def run_update_sweep(args, sampler=None, steps=None, settle_s=1.0):
         "config": {"workload": "c5: update-only sweep, Adam, 1e6..1e9 parameters in 1..500 log-uniform tensors",
                    "cache": "1e8 and 1e9 parameters (1.6 / 16 GB of state) far exceed the 126 MB L2",
                    "settle_s": settle_s},
-        "gpu_launches": int(mp.mp_kernel_launch_count() - launches0),
+        "gpu_launches": int(timed_launches),
         "roofline": {"kernel": "mp_master_update_kernel", "bound": "hbm", "achieved": top["gbs_28B"],
                      "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": top["gbs_28B"] / pk["hbm_gbs"],
                      "traffic": (NCU_UPDATE_TRAFFIC["bytes_per_param"] * top["params"]
@@ -470,9 +473,11 @@ def run_stack(args, name, steps, sampler, dist, full):
 
     def timed(fn, n, key=None, settle_s=None):
         """max over ranks of the device time of n calls, in ms, after the settling replays"""
+        t0 = time.time()            # the clock window covers the settling replays too: the same work, the same state
         s = settle(fn, args.settle if settle_s is None else settle_s, torch.cuda.synchronize)
         barrier()
-        t0 = time.time()
+        if s > 0.5:
+            t0 += 0.5               # without their first half second, in which the clocks still fall
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record()
         for _ in range(n):
@@ -576,11 +581,9 @@ def run_stack(args, name, steps, sampler, dist, full):
     # (D) the fused update alone, replayed back to back (last: it moves the weights without new
     # gradients, which nothing after it reads)
     if use_graph:
-        n0 = mp.mp_kernel_launch_count()
-        g_upd = stack.capture_only(xs, gs, ("update",))
-        n_launch = mp.mp_kernel_launch_count() - n0
-        ms, s = timed(g_upd.replay, steps, "update", args.settle / 2)
-        upd_only = (ms / steps / max(n_launch, 1), s)
+        ms, s = timed(lambda: mp.mp_master_update(stack.plan, stack.state, stack.opt, 0), steps, "update",
+                      args.settle / 2)
+        upd_only = (ms / steps, s)
     assert mp.mp_gemm_device_status() == 0, "a GEMM kernel reported a device-side error"
     assert stack.state.read().status == 0
 
@@ -654,7 +657,8 @@ def run_stack(args, name, steps, sampler, dist, full):
                      "frac_of_nominal_2250": gemm_tflops / 2250.0,
                      "sm_mhz_in_region": gemm_mhz, "clock_peak_tflops": clock_peak,
                      "frac_of_clock_peak": gemm_tflops / clock_peak if clock_peak else None,
-                     "clock_peak_how": f"{sms} SMs x {TENSOR_FLOP_PER_CLK_SM} flop/clk x median SM clock sampled inside this region",
+                     "clock_peak_how": f"{sms} SMs x {TENSOR_FLOP_PER_CLK_SM} flop/clk x median SM clock sampled inside this "
+                                       "region and the settling replays before it (nvidia-smi, every 50 ms)",
                      "launches": gemm_launches, "avg_launch_ms": gemm_ms / max(gemm_launches, 1),
                      "algorithmic_gflop_per_launch": flops_step * steps / max(gemm_launches, 1) / 1e9,
                      "algorithmic_mb_per_launch": cfg_gemm_bytes(cfg) * steps / max(gemm_launches, 1) / 1e6,
@@ -666,8 +670,9 @@ def run_stack(args, name, steps, sampler, dist, full):
                    "frac_of_nominal_8000": upd_gbs / 8000.0, "bytes_per_param": bytes_per_param,
                    "algorithmic_bytes_per_launch": upd_bytes,
                    "avg_launch_ms": upd_ms_alone, "peak_source": pk_src + " copy",
-                   "timed_in": ("the step's update call alone as a CUDA graph replayed back to back after settling "
-                                "replays" if upd_only is not None else timed_how),
+                   "timed_in": ("the step's update call alone, launched back to back (the kernel outlasts the host's "
+                                "call, so the launches queue without gaps) after settling launches"
+                                if upd_only is not None else timed_how),
                    "in_step": {"avg_launch_ms": upd_ms_in_step, "achieved": upd_bytes / (upd_ms_in_step * 1e-3) / 1e9,
                                "note": "between event nodes inside the step, right after the products"},
                    "traffic": (NCU_UPDATE_TRAFFIC["bytes_per_param"] * cfg.n_params()
@@ -735,7 +740,7 @@ def main():
     torch.cuda.set_device(local)
     if args.workload == "c5":
         if rank == 0:
-            print(json.dumps(run_update_sweep(args)))
+            print(json.dumps(run_update_sweep(args, settle_s=min(1.0, args.settle))))
         return
     if args.per_shape:
         args.workload = args.workload or "c2"

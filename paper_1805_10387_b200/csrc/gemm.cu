@@ -68,7 +68,8 @@ struct GroupMaps {
 
 struct GemmParams {
   int group;            // number of problems in this launch
-  int work_per_problem; // tiles x splits of one problem
+  int work_per_problem; // tiles x splits of one problem; within a problem the tile index runs fastest, so that the
+                        // CTAs running at one time work on the same slice of the reduction and share its panels in L2
   int Mo, No, R;        // output rows, output columns, reduction length
   int No8;              // No rounded down to a multiple of 8: the columns the output tensor map covers
   int m_tiles, n_tiles, splits, num_kb;
@@ -429,7 +430,7 @@ mp_gemm_kernel(const __grid_constant__ GroupMaps maps, const GemmParams p) {
     // (no_loads: the error-path self-test; nothing is issued, so nothing is in flight at exit)
     for (int w = blockIdx.x; w < total_work && ok && !p.no_loads; w += gridDim.x) {
       const int prob = w / p.work_per_problem, wl = w - prob * p.work_per_problem;
-      const int split = wl % p.splits, tile = wl / p.splits;
+      const int tiles = p.m_tiles * p.n_tiles, split = wl / tiles, tile = wl - split * tiles;
       const CUtensorMap* map_a = &maps.a[prob];
       const CUtensorMap* map_b = &maps.b[prob];
       const int m0 = tile_m(p, tile) * BM, n0 = tile_n(p, tile) * BN;
@@ -482,7 +483,7 @@ mp_gemm_kernel(const __grid_constant__ GroupMaps maps, const GemmParams p) {
     bool ok = true;
     for (int w = blockIdx.x; w < total_work && ok; w += gridDim.x, ++iter) {
       const int wl = w % p.work_per_problem;
-      const int split = wl % p.splits, tile = wl / p.splits;
+      const int tiles = p.m_tiles * p.n_tiles, split = wl / tiles, tile = wl - split * tiles;
       const uint32_t idesc =
           ptx::idesc_f16_f32(BM, tile_width(p.No, tile_n(p, tile) * BN), A_MN, B_MN);
       const int kb0 = (int)((int64_t)split * p.num_kb / p.splits);
@@ -531,7 +532,7 @@ mp_gemm_kernel(const __grid_constant__ GroupMaps maps, const GemmParams p) {
     bool ok = true;
     for (int w = blockIdx.x; w < total_work && ok; w += gridDim.x, ++iter) {
       const int prob = w / p.work_per_problem, wl = w - prob * p.work_per_problem;
-      const int split = wl % p.splits, tile = wl / p.splits;
+      const int tiles = p.m_tiles * p.n_tiles, split = wl / tiles, tile = wl - split * tiles;
       const int m0 = tile_m(p, tile) * BM, n0 = tile_n(p, tile) * BN;
       const int acc = iter & 1;
       const uint32_t acc_phase = (iter >> 1) & 1;
@@ -636,7 +637,7 @@ mp_gemm_pair_kernel(const __grid_constant__ GroupMaps maps, const GemmParams p) 
     bool ok = true;
     for (int w = pair; w < total_work && ok; w += npairs) {
       const int prob = w / p.work_per_problem, wl = w - prob * p.work_per_problem;
-      const int split = wl % p.splits, tile = wl / p.splits;
+      const int tiles = p.m_tiles * p.n_tiles, split = wl / tiles, tile = wl - split * tiles;
       const CUtensorMap* map_a = &maps.a[prob];
       const CUtensorMap* map_b = &maps.b[prob];
       const CUtensorMap* map_b32 = &maps.b32[prob];
@@ -705,7 +706,7 @@ mp_gemm_pair_kernel(const __grid_constant__ GroupMaps maps, const GemmParams p) 
       bool ok = true;
       for (int w = pair; w < total_work && ok; w += npairs, ++iter) {
         const int wl = w % p.work_per_problem;
-        const int split = wl % p.splits, tile = wl / p.splits;
+        const int tiles = p.m_tiles * p.n_tiles, split = wl / tiles, tile = wl - split * tiles;
         const uint32_t idesc =
             ptx::idesc_f16_f32(256, tile_width(p.No, tile_n(p, tile) * BN), A_MN, B_MN);
         const int kb0 = (int)((int64_t)split * p.num_kb / p.splits);
@@ -751,7 +752,7 @@ mp_gemm_pair_kernel(const __grid_constant__ GroupMaps maps, const GemmParams p) 
     bool ok = true;
     for (int w = pair; w < total_work && ok; w += npairs, ++iter) {
       const int prob = w / p.work_per_problem, wl = w - prob * p.work_per_problem;
-      const int split = wl % p.splits, tile = wl / p.splits;
+      const int tiles = p.m_tiles * p.n_tiles, split = wl / tiles, tile = wl - split * tiles;
       const int m0 = tile_m(p, tile) * 256 + 128 * (int)rank, n0 = tile_n(p, tile) * BN;
       const int acc = iter & 1;
       const uint32_t acc_phase = (iter >> 1) & 1;

@@ -24,6 +24,16 @@ def _bits(t):
     return t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
 
 
+def _rel_floor(red):
+    """The stated bar, max relative error 1e-2 against the FP32-accumulated oracle, is applied to
+    outputs of at least this fraction of the tensor's rms.  Both sides add the same exact products
+    in FP32 but in different orders; over a reduction of `red` terms that moves a sum by about
+    sqrt(red) * 2^-24 times the size of its partial sums (the rms), i.e. by 1e-2 of an output
+    that cancelled down to ~1e-4 * sqrt(red) of the rms.  Smaller outputs are covered by the
+    absolute bound above, which always holds."""
+    return max(1e-3, 1e-4 * float(red) ** 0.5)
+
+
 def _check_samples(orc, op, A, B, got, n_samples, seed):
     R, Cc = got.shape
     rng = np.random.default_rng(seed)
@@ -41,7 +51,7 @@ def _check_samples(orc, op, A, B, got, n_samples, seed):
     assert np.isinf(g[over]).all() and (np.sign(g[over]) == np.sign(ex[over])).all()
     fin = sure & (np.abs(w) > 2.0 ** -14)
     rms = np.sqrt((w[fin] ** 2).mean())
-    big = fin & (np.abs(w) >= 1e-3 * rms)
+    big = fin & (np.abs(w) >= _rel_floor(red) * rms)
     assert (np.abs(g[big] - w[big]) / np.abs(w[big])).max() <= 1e-2
     return float((got[rows, cols] == want16).mean())
 
@@ -255,7 +265,7 @@ def _check_product_samples(orc, op, A, B, got, n_samples, seed, what):
     fin = sure & (np.abs(w) > 2.0 ** -14)
     if fin.any():
         rms = np.sqrt((w[fin] ** 2).mean())
-        big = fin & (np.abs(w) >= 1e-3 * rms)
+        big = fin & (np.abs(w) >= _rel_floor(red) * rms)
         assert (np.abs(g[big] - w[big]) / np.abs(w[big])).max() <= 1e-2, what
     return float((got[rows, cols] == want16).mean())
 
@@ -327,7 +337,8 @@ def _update_check_streamed(orc, cfg, stack, pre, S, t_applied, chunk=1 << 23):
 def test_full_step(orc, mp, name, max_steps, want_applied):
     """Steps of the full-size workload, the first launched call by call, the rest replayed from the
     CUDA graph, until `want_applied` steps have been applied (the configured initial loss scale
-    overflows at first, so the first steps are skipped ones).  Every step: the flag against an
+    overflows at first on c2 and c4, so their first steps are skipped ones; c3 gets a planted inf
+    after its applied steps).  Every step: the flag against an
     independent scan of the stored weight gradients, scale and counters bit-exact against the
     scalar oracle, a skipped step leaves everything bitwise unchanged, an applied step's update
     is checked over the whole parameter range.  On the first step and on every applied step all
@@ -339,7 +350,15 @@ def test_full_step(orc, mp, name, max_steps, want_applied):
     sc = orc.Scaler(cfg.init_scale, cfg.growth_interval)
     applied = skipped = 0
     identical = []
-    for step in range(max_steps):
+    planted = None
+    for step in range(max_steps + 1):
+        if applied >= want_applied:
+            if skipped >= 1:
+                break
+            # no natural overflow at this workload's initial scale: plant one non-finite value in
+            # the gradient entering the last top layer, so that the skip runs at full size too
+            planted = [l for l in range(L) if not cfg.feeds_next(l)][-1]
+            gs[planted][0, 0] = float("inf")
         pre = (stack.w32_flat.clone(), stack.m_flat.clone(),
                stack.v_flat.clone() if stack.v_flat is not None else None)
         w16_pre = stack.w16_flat.clone()
@@ -375,7 +394,7 @@ def test_full_step(orc, mp, name, max_steps, want_applied):
                 Xg, dYg = _bits(stack.X(l)), _bits(stack.dY(l))
                 if not cfg.chained(l):
                     assert (Xg == xh[l]).all()
-                if not cfg.feeds_next(l):                   # upstream scaling: bitwise, whole tensor
+                if not cfg.feeds_next(l) and planted is None:   # upstream scaling: bitwise, whole tensor
                     assert (dYg == orc.scale_upstream(gh[l], S)).all()
                 n = 3400
                 same = [_check_product_samples(orc, "fwd", Xg, W, _bits(stack.Y(l)), n, 100 * l + step, f"Y{l} step {step}"),
@@ -396,7 +415,8 @@ def test_full_step(orc, mp, name, max_steps, want_applied):
             frac = _update_check_streamed(orc, cfg, stack, pre, S, t_pre + 1)
             assert frac > 0.99, frac                        # nearly every FP32 word bitwise equal
         del pre, w16_pre
-        if applied >= want_applied:
+        if planted is not None:
+            assert scan == 1
             break
     assert applied >= want_applied, (applied, skipped)
     assert skipped >= 1                                      # the halving path ran at full size too

@@ -28,6 +28,8 @@ def _bits(t):
 def test_static_scratch_matches_workspace_entry_point_twice(mp, M, K, N):
     need = mp.mp_gemm_workspace_bytes(M, K, N, mp.MP_OP_WGRAD)
     assert need <= mp.mp_static_scratch_bytes() == 32 << 20
+    if M >= 3000:
+        assert need > 0                           # these sizes really go through the scratch
     ws = torch.empty(max(need, 16), dtype=torch.uint8, device="cuda")
     for call in range(2):                         # second call: different data, stale scratch
         X = _rand16((M, K), 10 + call)
