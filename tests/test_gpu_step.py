@@ -16,6 +16,10 @@ def _f(bits):
     return bits.view(np.float16).astype(np.float64)
 
 
+def _h16(x):
+    return np.ascontiguousarray(x, np.float32).astype(np.float16).view(np.uint16)
+
+
 def _pad_dev(bits):
     r, c = bits.shape
     buf = torch.zeros(r, (c + 7) // 8 * 8, dtype=torch.float16, device="cuda")
@@ -395,3 +399,48 @@ def test_layers_with_bias_and_activation(orc, mp, name, shapes, acts, clip):
     cfg.growth_interval = 2
     recs = run_config(orc, mp, cfg, 4, acts=acts, bias=True, clip=clip)
     assert len(recs) == 4
+
+
+def test_weight_gradients_on_a_second_stream_change_nothing(orc, mp):
+    """The stack issues its weight-gradient products on a second stream (beside the data gradients
+    of the layers below).  Same kernels on the same operands: gradients, masters, moments, weights
+    and the loss-scale state are bit for bit those of the one-stream order, eagerly and replayed
+    from a CUDA graph, over steps that include a skipped one."""
+    from paper_1805_10387_b200.stack import LinearStack
+    shapes = [(384, 136, 520), (384, 520, 136), (384, 136, 136), (384, 136, 136)]   # chained pair + a group of two
+    chain = [False, True, False, False]
+    rng = np.random.default_rng(5)
+    ws = [rng.standard_normal((k, n)).astype(np.float32) / np.sqrt(k) for _, k, n in shapes]
+
+    def make(overlap):
+        st = LinearStack(shapes, chain, lr=1e-3, init_scale=2.0 ** 10, growth_interval=2, bias=True,
+                         acts=[mp.MP_ACT_RELU, 0, 0, 0], overlap_wgrad=overlap)
+        for l, w in enumerate(ws):
+            b = np.linspace(-0.1, 0.1, shapes[l][2]).astype(np.float32)
+            st.load_weights(l, torch.from_numpy(w).cuda(), torch.from_numpy(w).cuda().half(),
+                            torch.from_numpy(b).cuda(), torch.from_numpy(b).cuda().half())
+        return st
+    a, b, c = make(False), make(True), make(True)
+    assert b.side is not None and a.side is None and len(b.groups) == 3
+    xs = [_pad_dev(_h16(rng.standard_normal((m, k)))) if not chain[l] else None for l, (m, k, _) in enumerate(shapes)]
+    gs = [None] + [torch.from_numpy((rng.standard_normal((m, n)) * 1e-2).astype(np.float32)).cuda()
+                   for (m, _, n) in shapes[1:]]
+    c.capture(xs, gs, warmup=0)
+    for s in range(6):
+        if s == 3:
+            gs[2][0, 0] = float("inf")
+        if s == 4:
+            gs[2][0, 0] = 0.0
+        a.step(xs, gs); b.step(xs, gs); c.replay()
+    torch.cuda.synchronize()
+    assert mp.mp_gemm_device_status() == 0
+    ha = a.state.read()
+    assert ha.skipped == 1 and ha.step == 6
+    for o in (b, c):
+        h = o.state.read()
+        assert (h.scale, h.t, h.skipped, h.step, h.good_steps) == (ha.scale, ha.t, ha.skipped, ha.step, ha.good_steps)
+        for fa, fo in ((a.w32_flat, o.w32_flat), (a.m_flat, o.m_flat), (a.v_flat, o.v_flat)):
+            assert torch.equal(fa.view(torch.int32), fo.view(torch.int32))
+        assert torch.equal(a.w16_flat.view(torch.int16), o.w16_flat.view(torch.int16))
+        assert torch.equal(a.dw_flat.view(torch.int16), o.dw_flat.view(torch.int16))
+    a.close(); b.close(); c.close()
