@@ -40,7 +40,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # + dram__bytes_write.sum summed over one step's product launches, split-reduction kernels included,
 # divided by their number; on c2 a launch holds four layers' products, 4 x 95.4 MB algorithmic), valid
 # only for the kernel source it was taken on.
-NCU_TRAFFIC = {"sha": "0874106332883409", "bytes_per_launch": {"c2": 402.4e6, "c3": 82.3e6, "c4": 116.2e6}}
+NCU_TRAFFIC = {"sha": "0874106332883409", "bytes_per_launch": {"c2": 402.4e6, "c3": 176.9e6, "c4": 115.9e6}}
 # flop per clock and SM of the FP16 tensor pipe (one 128 x 256 x 16 MMA per SM in 128 clocks)
 TENSOR_FLOP_PER_CLK_SM = 8192
 
@@ -157,6 +157,15 @@ def oracle_sample_step(orc, synth, cfg, rows, upd_params, data=None):
     return t1 - t0, t2 - t1, 3 * 2 * rows * K * N, n * (28 if cfg.optimizer == "adam" else 20), data
 
 
+def workload_config(cfg, world=1, layers_kind="plain linear", sharded=False):
+    """The `config` object of the JSON line: the same for the CUDA arm and the reference arm."""
+    return {"workload": cfg.name + ": " + cfg.note, "layers": len(cfg.shapes), "params": cfg.n_params(),
+            "gemm_gflop_per_step": cfg.gemm_flops() / 1e9, "optimizer": cfg.optimizer,
+            "parallelism": (f"dp{world}" + (" sharded update" if sharded else "")) if world > 1 else "single",
+            "layers_kind": layers_kind,
+            "cache": "per-step working set (weights, moments, activations) far exceeds the 126 MB L2"}
+
+
 def cpu_baseline_of(orc, synth, cfg, seconds):
     """The oracle as it stands on the host cores, on a bounded sample of the workload: products and
     update timed apart (GFLOP/s, GB/s) and together (`value`, the whole-sample analogue of the
@@ -208,23 +217,37 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": val, "unit": "TFLOP/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": tot / args.steps * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f16 in / f32 accumulate",
-        "data": "synthetic", "config": {"workload": cfg.name + ": " + cfg.note},
+        "data": "synthetic", "config": workload_config(cfg),
         "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": sample,
                          "gemm_gflops": flops / tg / 1e9, "update_gbs": nbytes / tu / 1e9},
         "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
 
 
-def settle(fn, seconds, sync):
+def settle(fn, seconds, sync, dist=None):
     """Runs fn back to back, untimed, for about `seconds` of wall time so that the timed region
-    that follows starts in the power and clock state the same work settles into."""
+    that follows starts in the power and clock state the same work settles into.  With several
+    ranks every rank must make the same number of calls (fn holds collectives), so the count is
+    fixed from a short calibration and agreed on across the ranks."""
     t0 = time.time()
-    n = 0
-    while time.time() - t0 < seconds:
-        for _ in range(8):
-            fn()
-        n += 8
-        sync()
+    if seconds <= 0:
+        return 0.0
+    if dist is None:
+        while time.time() - t0 < seconds:
+            for _ in range(8):
+                fn()
+            sync()
+        return time.time() - t0
+    import torch
+    for _ in range(8):
+        fn()
+    sync()
+    per_call = max((time.time() - t0) / 8, 1e-5)
+    n = torch.tensor([int(seconds / per_call) + 1], device="cuda")
+    dist.all_reduce(n, op=dist.ReduceOp.MAX)
+    for _ in range(int(n.item())):
+        fn()
+    sync()
     return time.time() - t0
 
 
@@ -425,7 +448,8 @@ def run_stack(args, name, steps, sampler, dist, full):
     stack = LinearStack(cfg.shapes, chained, optimizer=cfg.optimizer, lr=cfg.lr, beta1=cfg.beta1,
                         beta2=cfg.beta2, eps=cfg.eps, momentum=cfg.momentum, init_scale=cfg.init_scale,
                         growth_interval=cfg.growth_interval, acts=acts, bias=args.real_layers and lstm is None,
-                        lstm=lstm, comm=comm, shard_update=args.shard_update)
+                        lstm=lstm, comm=comm, shard_update=args.shard_update,
+                        overlap_wgrad={"auto": None, "on": True, "off": False}[args.overlap_wgrad])
     gen = torch.Generator(device="cuda")
     gen.manual_seed(1234 + cfg.seed)           # same weights on every rank
     for l, (M, K, N) in enumerate(cfg.shapes):
@@ -474,7 +498,7 @@ def run_stack(args, name, steps, sampler, dist, full):
     def timed(fn, n, key=None, settle_s=None):
         """max over ranks of the device time of n calls, in ms, after the settling replays"""
         t0 = time.time()            # the clock window covers the settling replays too: the same work, the same state
-        s = settle(fn, args.settle if settle_s is None else settle_s, torch.cuda.synchronize)
+        s = settle(fn, args.settle if settle_s is None else settle_s, torch.cuda.synchronize, dist)
         barrier()
         if s > 0.5:
             t0 += 0.5               # without their first half second, in which the clocks still fall
@@ -536,7 +560,7 @@ def run_stack(args, name, steps, sampler, dist, full):
                 done.synchronize()
                 for nm, a, b in ev:
                     per.setdefault(nm, []).append(a.elapsed_time(b))
-        settle(stack.replay, args.settle / 2, torch.cuda.synchronize)
+        settle(stack.replay, args.settle / 2, torch.cuda.synchronize, dist)
         barrier()
         a_t, b_t = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a_t.record(); timed_steps(); b_t.record(); barrier()
@@ -631,15 +655,11 @@ def run_stack(args, name, steps, sampler, dist, full):
         "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f16 in / f32 accumulate", "data": "synthetic",
-        "config": {"workload": cfg.name + ": " + cfg.note, "layers": L, "params": cfg.n_params(),
-                   "gemm_gflop_per_step": flops_step / 1e9, "optimizer": cfg.optimizer,
-                   "parallelism": (f"dp{world}" + (" sharded update" if stack.shard_update else "")) if world > 1 else "single",
-                   "layers_kind": ("LSTM cells on the gate products" if lstm is not None else
-                                   "bias + activation (fused epilogues) + bias gradients" if args.real_layers
-                                   else "plain linear"),
-                   "cache": "per-step working set (weights, moments, activations) far exceeds the 126 MB L2",
-                   "settle_s": settle_step,
-                   "settle": "every device-timed region follows that many seconds of untimed replays of itself"},
+        "config": workload_config(cfg, world, "LSTM cells on the gate products" if lstm is not None else
+                                  "bias + activation (fused epilogues) + bias gradients" if args.real_layers
+                                  else "plain linear", stack.shard_update),
+        "settle_s": settle_step,
+        "settle": "every device-timed region follows that many seconds of untimed replays of itself",
         "gpu_launches": int(launches),
         "launch_mode": "one CUDA graph replay per step (captured from the same C-ABI calls)" if use_graph
                        else "call by call",
@@ -727,6 +747,8 @@ def main():
     ap.add_argument("--shard-update", action="store_true",
                     help="several GPUs: reduce-scatter the gradients, update a 1/N slice of the master per rank, "
                          "all-gather the FP16 weights (default: all-reduce and a replicated update)")
+    ap.add_argument("--overlap-wgrad", default="auto", choices=["auto", "on", "off"],
+                    help="weight gradients on a second stream beside the data gradients (auto: stacks with chained layers)")
     ap.add_argument("--max-params", type=float, default=1e9, help="c5: largest parameter count of the sweep")
     args = ap.parse_args()
     if args.impl == "reference":

@@ -153,21 +153,25 @@ class LinearStack:
                 self.dy[l] = self.dy_top_flat[flat_off[l]:flat_off[l] + m * n].view(m, n)
             else:
                 self.dy[l] = torch.zeros(self.shapes[l][0], _align(self.shapes[l][2]), **f16)
-        # Runs of consecutive layers that depend on nothing in the stack (no chained input, output
-        # feeding no layer), have one shape and no activation go to the grouped calls, a few
-        # layers per launch; every other layer is a group of one.
-        self.groups = []
+        # Launch groups.  A layer's level is its depth in its chain (0 for a layer that reads an input of
+        # the stack).  Layers of one level do not depend on one another, so those of them that have one
+        # shape, one activation and the same kind of neighbours go to the grouped calls, a few layers per
+        # launch: a product too small to fill the GPU's waves on its own then shares a persistent work
+        # list with its peers.  Forward runs the groups level by level, backward in the reverse order.
         gmax = mp.mp_max_group()
+        level = [0] * self.L
         for l in range(self.L):
-            free = (not self.chained[l] and not (l + 1 < self.L and self.chained[l + 1])
-                    and self.acts[l] == mp.MP_ACT_NONE)
-            g = self.groups[-1] if self.groups else None
-            if (free and g is not None and g[1] and len(g[0]) < gmax
-                    and self.shapes[g[0][0]] == self.shapes[l]):
-                g[0].append(l)
-            else:
-                self.groups.append(([l], free))
-        self.groups = [g[0] for g in self.groups]
+            level[l] = level[l - 1] + 1 if self.chained[l] else 0
+        buckets = {}
+        for l in range(self.L):
+            below = self.acts[l - 1] if self.chained[l] else mp.MP_ACT_NONE
+            key = (level[l], self.shapes[l], self.acts[l], self.lstm[l], self.chained[l], self.feeds_next(l), below)
+            buckets.setdefault(key, []).append(l)
+        self.groups = []
+        for key in sorted(buckets, key=lambda k: (k[0], buckets[k][0])):
+            ls = buckets[key]
+            for i in range(0, len(ls), gmax):
+                self.groups.append(ls[i:i + gmax])
         need = 0
         for g in self.groups:
             m, k, n = self.shapes[g[0]]
@@ -183,8 +187,9 @@ class LinearStack:
         # them), and a persistent product kernel leaves SMs idle in its last, partly filled wave of
         # tiles: issued on a second stream, a weight gradient's CTAs take the SMs that the data gradient
         # before it has already left, and vice versa.  The second stream has a workspace of its own.
-        # Measured (settled bench, whole step): c3 3.92 -> 3.85 ms, c4 2.01 -> 1.97 ms; c2, whose launches are
-        # all full-size and independent, 2.49 -> 2.52 ms (hence the default).
+        # Measured on one B200 (whole step, alternating runs): the Transformer-like stack 3.93 -> 3.86 ms, the
+        # DeepSpeech2-like chain 1.99 -> 1.955 ms; a stack of independent full-size layers 2.49 -> 2.52 ms
+        # (hence the default).
         self.overlap_wgrad = any(self.chained) if overlap_wgrad is None else bool(overlap_wgrad)
         self.side = torch.cuda.Stream(device=self.device) if self.overlap_wgrad else None
         self.workspace_side = torch.empty(max(need, 16), dtype=torch.uint8, device=self.device) \
@@ -390,8 +395,11 @@ class LinearStack:
             if len(g) > 1 and len({self.x[l].stride(0) for l in g}) == 1:
                 if self.has_bias:
                     self._call("fwd", mp.mp_linear_fwd_act_grouped, [Xv(l) for l in g], [self.W16(l) for l in g],
-                               [self.b16[l] for l in g], [self.Y(l) for l in g], mp.MP_ACT_NONE, self.clip,
+                               [self.b16[l] for l in g], [self.Y(l) for l in g], self.acts[g[0]], self.clip,
                                self.workspace)
+                elif self.acts[g[0]] != mp.MP_ACT_NONE:
+                    self._call("fwd", mp.mp_linear_fwd_act_grouped, [Xv(l) for l in g], [self.W16(l) for l in g],
+                               None, [self.Y(l) for l in g], self.acts[g[0]], self.clip, self.workspace)
                 else:
                     self._call("fwd", mp.mp_linear_fwd_grouped, [Xv(l) for l in g], [self.W16(l) for l in g],
                                [self.Y(l) for l in g], self.workspace)
@@ -425,34 +433,32 @@ class LinearStack:
                 if self.lstm[l]:      # gradient of h -> gradient of the gate pre-activations
                     self._call("cell", mp.mp_lstm_cell_bwd, self.Y(l), self.c_prev[l], self.c_new[l], self.dh[l],
                                None, self.dY(l), self.dc_prev[l])
-            if (len(g) > 1 and len({self.x[l].stride(0) for l in g}) == 1
-                    and len({self.dy[l].stride(0) for l in g}) == 1):
-                self._fork()                               # the group's dY is complete
-                with self._wgrad_stream():
+            grouped = (len(g) > 1 and len({self.x[l].stride(0) for l in g}) == 1
+                       and len({self.dy[l].stride(0) for l in g}) == 1)
+            # the activation of the layer below (the same for every layer of a group) masks the data gradient
+            below = self.acts[g[0] - 1] if self.chained[g[0]] else mp.MP_ACT_NONE
+            self._fork()                                   # the group's dY is complete
+            with self._wgrad_stream():
+                if grouped:
                     self._call("wgrad", mp.mp_linear_bwd_wgrad_grouped, [Xv(l) for l in g], [self.dY(l) for l in g],
                                [self.dW(l) for l in g], self.state, self.workspace_side)
+                for l in reversed(g):
+                    if not grouped:
+                        self._call("wgrad", mp.mp_linear_bwd_wgrad, Xv(l), self.dY(l), self.dW(l), self.state,
+                                   self.workspace_side)
                     if self.has_bias:
-                        for l in reversed(g):
-                            self._call("bgrad", mp.mp_bias_grad, self.dY(l), self.db[l], self.state,
-                                       self.workspace_side)
+                        self._call("bgrad", mp.mp_bias_grad, self.dY(l), self.db[l], self.state,
+                                   self.workspace_side)
+            if grouped and below == mp.MP_ACT_NONE:
                 self._call("dgrad", mp.mp_linear_bwd_dgrad_grouped, [self.dY(l) for l in g],
                            [self.W16(l) for l in g], [self.dX(l) for l in g], self.workspace)
                 continue
             for l in reversed(g):
-                X = Xv(l)
-                self._fork()                               # this layer's dY is complete
-                with self._wgrad_stream():
-                    self._call("wgrad", mp.mp_linear_bwd_wgrad, X, self.dY(l), self.dW(l), self.state,
-                               self.workspace_side)
-                    if self.has_bias:
-                        self._call("bgrad", mp.mp_bias_grad, self.dY(l), self.db[l], self.state,
-                                   self.workspace_side)
-                below = self.acts[l - 1] if self.chained[l] else mp.MP_ACT_NONE
                 if below == mp.MP_ACT_NONE:
                     self._call("dgrad", mp.mp_linear_bwd_dgrad, self.dY(l), self.W16(l), self.dX(l),
                                self.workspace)
                 else:   # the layer below is activated: mask with its stored output (= this layer's input)
-                    self._call("dgrad", mp.mp_linear_bwd_dgrad_act, self.dY(l), self.W16(l), X, self.dX(l),
+                    self._call("dgrad", mp.mp_linear_bwd_dgrad_act, self.dY(l), self.W16(l), Xv(l), self.dX(l),
                                below, self.clip, self.workspace)
         self._join()                                       # every weight gradient is complete
 
