@@ -46,9 +46,9 @@ TENSOR_FLOP_PER_CLK_SM = 8192
 
 
 # DRAM bytes per parameter of the fused update from one ncu capture at 1e8 parameters in 64 tensors
-# (2.7406 GB per launch); a launch over P parameters moves P times this (traffic grows in
+# (2.7404 GB per launch); a launch over P parameters moves P times this (traffic grows in
 # proportion: every parameter is touched once), valid only for the kernel source it was taken on.
-NCU_UPDATE_TRAFFIC = {"sha": "3718ba9d82009239", "bytes_per_param": 27.41}
+NCU_UPDATE_TRAFFIC = {"sha": "77306490e753c3d8", "bytes_per_param": 27.40}
 
 
 def update_kernel_sha():

@@ -245,6 +245,11 @@ int mp_linear_bwd_dgrad_act(const void* dY16, int64_t lddy, const void* W16, int
 int mp_bias_grad(const void* dY16, int64_t lddy, void* db16, int64_t M, int64_t N, mp_state* state,
                  void* workspace, size_t workspace_bytes, void* stream);
 size_t mp_bias_grad_workspace_bytes(int64_t M, int64_t N);
+/* The same for `count` (1 .. mp_max_group()) gradients of one shape and row pitch in one pair of launches: dY16 and
+ * db16 are host arrays of `count` device pointers; every result is the single call's, bit for bit.
+ * workspace: at least count * mp_bias_grad_workspace_bytes(M,N) bytes. */
+int mp_bias_grad_grouped(int count, const void* const* dY16, int64_t lddy, void* const* db16, int64_t M,
+                         int64_t N, mp_state* state, void* workspace, size_t workspace_bytes, void* stream);
 
 /* LSTM cell for a gate product G = [x;h] W of 4H columns in the order i, f, g, o (the GNMT-like
  * layers of Section 5; the paper gives no arithmetic, so: FP16 gates and states in memory, the

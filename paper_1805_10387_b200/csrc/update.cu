@@ -335,9 +335,16 @@ mp_scale_upstream_kernel(const float* __restrict__ g32, uint16_t* __restrict__ o
 // below N lies inside its row; columns at or beyond N are read and dropped.
 constexpr int kBiasSlabs = 512;
 constexpr int kBiasCols = 256;
+constexpr int kBiasGroup = 4;      // gradients of one shape that may share a launch (blockIdx.z picks one)
+struct BiasGroup {
+  const uint16_t* dY[kBiasGroup];
+  uint16_t* db[kBiasGroup];
+};
 __global__ void __launch_bounds__(kThreads, 8)
-mp_bias_grad_partial_kernel(const uint16_t* __restrict__ dY, int64_t lddy, int64_t M, int64_t N,
-                            float* __restrict__ partial, int slabs, int vecs) {
+mp_bias_grad_partial_kernel(const BiasGroup group, int64_t lddy, int64_t M, int64_t N,
+                            float* __restrict__ partial_all, int slabs, int vecs) {
+  const uint16_t* __restrict__ dY = group.dY[blockIdx.z];
+  float* __restrict__ partial = partial_all + (int64_t)blockIdx.z * slabs * N;
   // vecs: vectors per row handled by one warp, a power of two <= 32
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int groups = 32 / vecs;                     // rows a warp reads at once
@@ -393,8 +400,10 @@ mp_bias_grad_partial_kernel(const uint16_t* __restrict__ dY, int64_t lddy, int64
 // order through shared memory.
 constexpr int kBiasFinalThreads = 1024;
 __global__ void __launch_bounds__(kBiasFinalThreads)
-mp_bias_grad_final_kernel(const float* __restrict__ partial, int slabs, int64_t N,
-                          uint16_t* __restrict__ db, mp_dev_state* st) {
+mp_bias_grad_final_kernel(const float* __restrict__ partial_all, int slabs, int64_t N,
+                          const BiasGroup group, mp_dev_state* st) {
+  const float* __restrict__ partial = partial_all + (int64_t)blockIdx.y * slabs * N;
+  uint16_t* __restrict__ db = group.db[blockIdx.y];
   const int lane = threadIdx.x & 31, grp = threadIdx.x >> 5;
   const int64_t n = (int64_t)blockIdx.x * 32 + lane;
   const int per = (slabs + 31) / 32;
@@ -762,24 +771,33 @@ size_t mp_bias_grad_workspace_bytes(int64_t M, int64_t N) {
   return (size_t)bias_slabs(M, N) * (size_t)N * sizeof(float);
 }
 
-int mp_bias_grad(const void* dY16, int64_t lddy, void* db16, int64_t M, int64_t N, mp_state* state,
-                 void* workspace, size_t workspace_bytes, void* stream) {
-  if (!dY16 || !db16 || M <= 0 || N <= 0 || lddy < N)
-    return mp::set_error(MP_ERR_INVALID_ARG, "mp_bias_grad: bad argument");
-  if (!mp::aligned16(dY16) || !mp::aligned16(db16) || (lddy & 7) || (workspace && !mp::aligned16(workspace)))
+int mp_bias_grad_grouped(int count, const void* const* dY16, int64_t lddy, void* const* db16, int64_t M,
+                         int64_t N, mp_state* state, void* workspace, size_t workspace_bytes, void* stream) {
+  if (count < 1 || count > kBiasGroup || !dY16 || !db16 || M <= 0 || N <= 0 || lddy < N)
+    return mp::set_error(MP_ERR_INVALID_ARG, "mp_bias_grad: bad argument (1..%d gradients per call)", kBiasGroup);
+  for (int i = 0; i < count; ++i) {
+    if (!dY16[i] || !db16[i]) return mp::set_error(MP_ERR_INVALID_ARG, "mp_bias_grad: null pointer");
+    if (!mp::aligned16(dY16[i]) || !mp::aligned16(db16[i]))
+      return mp::set_error(MP_ERR_ALIGNMENT, "mp_bias_grad: buffers must be 16-byte aligned");
+  }
+  if ((lddy & 7) || (workspace && !mp::aligned16(workspace)))
     return mp::set_error(MP_ERR_ALIGNMENT, "mp_bias_grad: buffers must be 16-byte aligned, lddy a multiple of 8");
-  const size_t need = mp_bias_grad_workspace_bytes(M, N);
+  const size_t need = (size_t)count * mp_bias_grad_workspace_bytes(M, N);
   if (!workspace || workspace_bytes < need)
     return mp::set_error(MP_ERR_NOMEM, "mp_bias_grad: workspace of %zu bytes needed", need);
   if (int rc = mp::check_device()) return rc;
   const int slabs = bias_slabs(M, N);
   cudaStream_t st = (cudaStream_t)stream;
-  const dim3 grid((unsigned)((N + kBiasCols - 1) / kBiasCols), (unsigned)slabs);
+  BiasGroup grp;
+  for (int i = 0; i < kBiasGroup; ++i) {
+    grp.dY[i] = (const uint16_t*)dY16[i < count ? i : 0];
+    grp.db[i] = (uint16_t*)db16[i < count ? i : 0];
+  }
+  const dim3 grid((unsigned)((N + kBiasCols - 1) / kBiasCols), (unsigned)slabs, (unsigned)count);
   const int vecs = bias_vecs(N);
-  mp_bias_grad_partial_kernel<<<grid, kThreads, 0, st>>>((const uint16_t*)dY16, lddy, M, N,
-                                                        (float*)workspace, slabs, vecs);
+  mp_bias_grad_partial_kernel<<<grid, kThreads, 0, st>>>(grp, lddy, M, N, (float*)workspace, slabs, vecs);
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)((N + 31) / 32), 1, 1);
+  cfg.gridDim = dim3((unsigned)((N + 31) / 32), (unsigned)count, 1);
   cfg.blockDim = dim3(kBiasFinalThreads, 1, 1);
   cfg.stream = st;
   cudaLaunchAttribute attr;            // resident early, waits on the device for stage 1
@@ -788,9 +806,16 @@ int mp_bias_grad(const void* dY16, int64_t lddy, void* db16, int64_t M, int64_t 
   cfg.attrs = &attr;
   cfg.numAttrs = 1;
   MP_CUDA_TRY(cudaLaunchKernelEx(&cfg, mp_bias_grad_final_kernel,
-      (const float*)workspace, slabs, N, (uint16_t*)db16, state ? state->dev : (mp_dev_state*)nullptr));
+      (const float*)workspace, slabs, N, grp, state ? state->dev : (mp_dev_state*)nullptr));
   mp::count_launch(2);
   return MP_OK;
+}
+
+int mp_bias_grad(const void* dY16, int64_t lddy, void* db16, int64_t M, int64_t N, mp_state* state,
+                 void* workspace, size_t workspace_bytes, void* stream) {
+  const void* dys[1] = {dY16};
+  void* dbs[1] = {db16};
+  return mp_bias_grad_grouped(1, dys, lddy, dbs, M, N, state, workspace, workspace_bytes, stream);
 }
 
 int mp_check_finite(const void* g16, int64_t n, mp_state* state, void* stream) {

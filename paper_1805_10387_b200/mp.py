@@ -73,6 +73,7 @@ SIGNATURES = {
                                        C.c_float, _p, _sz, _p]),
     "mp_bias_grad": (_i32, [_p, _i64, _p, _i64, _i64, _p, _p, _sz, _p]),
     "mp_bias_grad_workspace_bytes": (_sz, [_i64, _i64]),
+    "mp_bias_grad_grouped": (_i32, [_i32, _p, _i64, _p, _i64, _i64, _p, _p, _sz, _p]),
     "mp_lstm_cell_fwd": (_i32, [_p, _i64, _p, _p, _p, _i64, _i64, _p]),
     "mp_lstm_cell_bwd": (_i32, [_p, _i64, _p, _p, _p, _p, _p, _i64, _p, _i64, _i64, _p]),
     "mp_master_update": (_i32, [_p, _p, C.POINTER(OptimConfig), _i32, _p]),
@@ -286,6 +287,15 @@ def mp_bias_grad(dY16, db16, state=None, workspace=None):
     ws, nb = _ws(workspace)
     _check(lib().mp_bias_grad(dy, lddy, _dev(db16, torch.float16), M, N,
                               state.handle if state is not None else None, ws, nb, _stream()))
+
+
+def mp_bias_grad_grouped(dY16s, db16s, state=None, workspace=None):
+    dy, lddy, (M, N) = _mats(dY16s)
+    assert len(db16s) == len(dY16s) and all(t.numel() == N and t.is_contiguous() for t in db16s)
+    db = (C.c_void_p * len(db16s))(*[_dev(t, torch.float16) for t in db16s])
+    ws, nb = _ws(workspace)
+    _check(lib().mp_bias_grad_grouped(len(dY16s), dy, lddy, db, M, N,
+                                      state.handle if state is not None else None, ws, nb, _stream()))
 
 
 def mp_lstm_cell_fwd(G16, c_prev16, c_new16, h16):

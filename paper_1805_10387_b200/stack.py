@@ -181,7 +181,7 @@ class LinearStack:
             for op in (mp.MP_OP_FWD, mp.MP_OP_DGRAD, mp.MP_OP_WGRAD):
                 need = max(need, mp.mp_gemm_workspace_bytes(m, k, n, op))
             if self.has_bias:
-                need = max(need, mp.mp_bias_grad_workspace_bytes(m, n))
+                need = max(need, gmax * mp.mp_bias_grad_workspace_bytes(m, n))
         self.workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=self.device)
         # The weight gradients are off the backward pass's critical path (nothing but the update reads
         # them), and a persistent product kernel leaves SMs idle in its last, partly filled wave of
@@ -442,13 +442,16 @@ class LinearStack:
                 if grouped:
                     self._call("wgrad", mp.mp_linear_bwd_wgrad_grouped, [Xv(l) for l in g], [self.dY(l) for l in g],
                                [self.dW(l) for l in g], self.state, self.workspace_side)
+                    if self.has_bias:
+                        self._call("bgrad", mp.mp_bias_grad_grouped, [self.dY(l) for l in g],
+                                   [self.db[l] for l in g], self.state, self.workspace_side)
                 for l in reversed(g):
                     if not grouped:
                         self._call("wgrad", mp.mp_linear_bwd_wgrad, Xv(l), self.dY(l), self.dW(l), self.state,
                                    self.workspace_side)
-                    if self.has_bias:
-                        self._call("bgrad", mp.mp_bias_grad, self.dY(l), self.db[l], self.state,
-                                   self.workspace_side)
+                        if self.has_bias:
+                            self._call("bgrad", mp.mp_bias_grad, self.dY(l), self.db[l], self.state,
+                                       self.workspace_side)
             if grouped and below == mp.MP_ACT_NONE:
                 self._call("dgrad", mp.mp_linear_bwd_dgrad_grouped, [self.dY(l) for l in g],
                            [self.W16(l) for l in g], [self.dX(l) for l in g], self.workspace)

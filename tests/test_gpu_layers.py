@@ -143,6 +143,33 @@ def test_bias_grad(orc, mp, M, N):
     st.close()
 
 
+def test_bias_grad_grouped_equals_single_calls(orc, mp):
+    """Four gradients of one shape in one pair of launches: every result is the single call's,
+    bit for bit, and the oracle's on integer values; a non-finite sum in one of them raises the flag."""
+    M, N = 777, 520
+    rng = np.random.default_rng(9)
+    dYs = [_h(rng.standard_normal((M, N)) * 3) for _ in range(3)] + [_h(rng.integers(-3, 4, (M, N)))]
+    devs = [_dev(d) for d in dYs]
+    single = [torch.zeros(N, dtype=torch.float16, device="cuda") for _ in dYs]
+    grouped = [torch.full((N,), 7.0, dtype=torch.float16, device="cuda") for _ in dYs]
+    ws = torch.empty(4 * mp.mp_bias_grad_workspace_bytes(M, N), dtype=torch.uint8, device="cuda")
+    st = mp.State()
+    for d, o in zip(devs, single):
+        mp.mp_bias_grad(d, o, st, ws)
+    mp.mp_bias_grad_grouped(devs, grouped, st, ws)
+    for a, b in zip(single, grouped):
+        assert torch.equal(a.view(torch.int16), b.view(torch.int16))
+    assert (_bits(grouped[3]) == orc.bias_grad(dYs[3])).all()
+    assert st.read().found_inf == 0
+    dYs[1][5, 17] = 0x7C00
+    mp.mp_bias_grad_grouped([_dev(d) for d in dYs], grouped, st, ws)
+    assert _bits(grouped[1])[17] == 0x7C00 and st.read().found_inf == 1
+    assert torch.equal(grouped[0].view(torch.int16), single[0].view(torch.int16))
+    with pytest.raises(mp.MpError):
+        mp.mp_bias_grad_grouped(devs, grouped, st, ws[:16])
+    st.close()
+
+
 # ------------------------------------------------------------------ LSTM cell
 @pytest.mark.parametrize("M,H", [(1, 8), (37, 64), (640, 1024)])
 def test_lstm_cell_forward_and_backward(orc, mp, M, H):
