@@ -170,6 +170,25 @@ def test_adam_against_library_float64(orc, wd):
     assert (w16 == _h(w32)).all()
 
 
+def test_weight_decay_is_formed_from_the_fp32_master(orc):
+    """Section 3.3: the decay term uses the FP32 master, not the FP16 working copy.  With a zero
+    gradient the only input of the step is wd * w, for weights that FP16 cannot hold exactly."""
+    w0 = np.array([1.0 + 2.0 ** -12, 3.0001, -0.3333333, 1e-9, 70000.0], np.float32)   # none is an FP16 value
+    assert (_h(w0).view(np.float16).astype(np.float32) != w0).all()
+    g0 = np.zeros(w0.size, np.uint16)
+    # momentum SGD with mu = 0, lr * wd = 1/2: every step halves the master exactly
+    w32 = w0.copy(); u = np.zeros_like(w0); w16 = np.zeros(w0.size, np.uint16)
+    for step in range(1, 4):
+        orc.momentum_update(g0, w32, u, w16, 1.0, 0.5, 0.0, 1.0)
+        assert (w32 == w0 * np.float32(0.5 ** step)).all()
+        assert (u == w0 * np.float32(0.5 ** (step - 1))).all()              # u = wd * w of the step
+    # Adam: the first moment is (1 - b1) * wd * w32 to FP32 rounding; from the FP16 copy it would be off by 2^-11
+    w32, m, v, w16 = _state(w0.size, w0)
+    orc.adam_update(g0, w32, m, v, w16, 1.0, t=1, weight_decay=0.5, **ADAM)
+    want = (1.0 - np.float64(np.float32(0.9))) * 0.5 * w0.astype(np.float64)
+    assert np.allclose(m, want, rtol=1e-6, atol=0)
+
+
 # -------------------------------------------------------------- momentum
 def test_momentum_constant_gradient_closed_form(orc):
     g = np.array([0.5, -0.125], np.float32)
