@@ -68,6 +68,28 @@ MUTANTS = [
      ["test_oracle_layers.py"]),
     ("only_the_bottom_layer_is_inspected", PY, "        flag |= found_inf(ly.dW)", "        flag = found_inf(ly.dW)",
      ["test_oracle_step.py"]),
+    ("f2h_nan_becomes_inf", CPP, "return (uint16_t)(sign | 0x7E00u);           // NaN",
+     "return (uint16_t)(sign | 0x7C00u);           // NaN", ["test_oracle_fp16.py"]),
+    ("h2f_nan_becomes_inf", CPP, "return bits_f32(sign | 0x7F800000u | (f << 13));", "return bits_f32(sign | 0x7F800000u);",
+     ["test_oracle_fp16.py", "test_oracle_matmul.py"]),
+    ("products_rounded_to_fp16", CPP,
+     "acc = acc + h2f(X[m * ldx + k]) * h2f(W[k * ldw + n]);\n        Y[m * ldy + n] = f2h(acc);",
+     "acc = acc + h2f(f2h(h2f(X[m * ldx + k]) * h2f(W[k * ldw + n])));\n        Y[m * ldy + n] = f2h(acc);",
+     ["test_oracle_matmul.py"]),
+    ("adam_first_moment_not_averaged", CPP, "const float mi = b1 * m[i] + omb1 * g;", "const float mi = b1 * m[i] + g;",
+     ["test_oracle_update.py"]),
+    ("static_scale_still_halves", CPP, "if (s->dynamic && s->strikes >= s->tolerance)", "if (s->strikes >= s->tolerance)",
+     ["test_oracle_update.py"]),
+    ("adam_step_count_off_by_one", PY, "        t = scaler.t + 1\n", "        t = scaler.t + 2\n", ["test_oracle_step.py"]),
+    ("sampled_wgrad_index", CPP, "else              { a = h2f(A[j * lda + r]); b = h2f(B[j * ldb + c]); }\n      acc = acc + a * b;",
+     "else              { a = h2f(A[j * lda + r]); b = h2f(B[c * ldb + j]); }\n      acc = acc + a * b;",
+     ["test_oracle_matmul.py"]),
+    ("exact_sum_drops_sign", CPP, "          ex += (double)a * (double)b;\n          ab += std::fabs((double)a * (double)b);\n        }\n        out_exact",
+     "          ex += std::fabs((double)a * (double)b);\n          ab += std::fabs((double)a * (double)b);\n        }\n        out_exact",
+     ["test_oracle_matmul.py"]),
+    ("exact_abs_sum_signed", CPP, "          ex += (double)a * (double)b;\n          ab += std::fabs((double)a * (double)b);\n        }\n        out_exact",
+     "          ex += (double)a * (double)b;\n          ab += (double)a * (double)b;\n        }\n        out_exact",
+     ["test_oracle_matmul.py"]),
     ("overflow_step_applied", PY, "    if not flag:                                          # Section 3.2",
      "    if True:", ["test_oracle_step.py"]),
     ("scale_applied_twice", PY, "ly.dY = layers[l + 1].dX if feeds_next else scale_upstream(gs[l], S)",

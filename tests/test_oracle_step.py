@@ -55,6 +55,31 @@ def test_c1_flags_skip_and_scale_trajectory(orc):
     assert sc.skipped == 1 and sc.t == 9
 
 
+def test_master_trajectory_matches_a_library_adam_fed_the_same_gradients(orc):
+    """The step driver's bookkeeping around the optimizer: the bias-correction count is the number of
+    APPLIED steps including the current one (first applied step: 1) and does not advance on a skipped
+    step.  A library Adam in float64 (an independent implementation) is stepped with the gradients the
+    oracle's step produced, unscaled, on applied steps only; the masters must follow it."""
+    import torch
+    cfg = synth.config("c1")
+    layers, sc, opt = _build(orc, cfg)
+    params = [torch.tensor(ly.w32.astype(np.float64), requires_grad=True) for ly in layers]
+    ref = torch.optim.Adam(params, lr=cfg.lr, betas=(cfg.beta1, cfg.beta2), eps=cfg.eps)
+    applied = 0
+    for step in range(8):                               # the inf arrives at step index 4
+        rec = orc.train_step(layers, *_inputs(cfg, step), sc, opt)
+        if rec.found_inf:
+            continue
+        applied += 1
+        for p, ly in zip(params, layers):
+            p.grad = torch.tensor(orc.h2f(ly.dW).astype(np.float64) / rec.S_before)
+        ref.step()
+        for p, ly in zip(params, layers):
+            want = p.detach().numpy()
+            assert np.abs(ly.w32 - want).max() <= 2e-6 * max(1.0, np.abs(want).max()), step
+    assert applied == 7 and sc.t == 7 and sc.skipped == 1
+
+
 def _dyadic_inputs(cfg, step):
     """Inputs on a dyadic grid: X integers in -2..2, upstream gradients multiples of 2^-5 in
     [-1/4, 1/4].  With weights on a 2^-4 grid every product sum is a multiple of 2^-9, so no
